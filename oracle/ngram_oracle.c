@@ -1,0 +1,309 @@
+/*
+ * CPU oracle for the batched N-gram speculation step ("The N-Grammys",
+ * arXiv 2411.03786).  TEST INFRASTRUCTURE ONLY: plain, slow, written for a
+ * reader to check against the paper by eye.  It shares no code with the CUDA
+ * library and the product never calls it.  Floating point is fp64 over the
+ * bf16-rounded inputs the tensor-core path also sees.
+ *
+ * Every routine is the definition written out; no blocking, no fusion.
+ * OpenMP, where present, only spreads independent rows / sequences over cores.
+ *
+ * Pins (tests/test_oracle_*.py): brute force on tiny inputs, a hand-worked
+ * example, closed forms (tied unit-norm weights, permutation weights),
+ * library matmul/unique cross-checks and the toy-model losslessness
+ * invariant.  No routine here is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------ bf16 storage */
+
+/* bfloat16 = the upper 16 bits of an IEEE binary32. */
+static double bf16_to_double(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+/* binary32 -> bfloat16, round to nearest, ties to even.  The Tiny configuration
+ * hands fp32 weights to a bf16 tensor-core path; both sides round once, like this. */
+uint16_t oracle_f32_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return (uint16_t)((u >> 16) | 0x40u); /* NaN */
+    uint32_t keep = u >> 16, rest = u & 0xFFFFu;
+    if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u))) keep += 1u;
+    return (uint16_t)keep;
+}
+
+void oracle_round_to_bf16(const float* in, uint16_t* out, long n) {
+    for (long i = 0; i < n; ++i) out[i] = oracle_f32_to_bf16(in[i]);
+}
+
+/* ------------------------------------------------------------------ context N-gram (Section 4.2)
+ *
+ * Query = the last q tokens of the history.  Every earlier full window of q+w
+ * tokens (stride 1, overlaps allowed) whose first q tokens equal the query is a
+ * match; the w tokens after it are its continuation.  Each distinct continuation
+ * gets count = number of matches and last = the largest window start among them.
+ * Order: count descending, ties by the later occurrence (last descending).
+ * Returns the number of rows written (<= topk).  rows is [topk, w].
+ */
+int oracle_context_draft(const int32_t* hist, int L, int q, int w, int topk,
+                         int32_t* rows, int32_t* counts, int32_t* lasts) {
+    if (q < 1 || w < 1 || topk < 1 || L < q + w) return 0;
+    const int32_t* query = hist + (L - q);
+    int n_windows = L - q - w + 1;
+    int* g_first = (int*)malloc(sizeof(int) * (size_t)n_windows); /* a window start representing the group */
+    int* g_count = (int*)malloc(sizeof(int) * (size_t)n_windows);
+    int* g_last = (int*)malloc(sizeof(int) * (size_t)n_windows);
+    char* g_taken = (char*)calloc((size_t)n_windows, 1);
+    int n_groups = 0;
+    for (int i = 0; i < n_windows; ++i) {
+        int match = 1;
+        for (int t = 0; t < q; ++t)
+            if (hist[i + t] != query[t]) { match = 0; break; }
+        if (!match) continue;
+        const int32_t* c = hist + i + q;
+        int g = -1;
+        for (int j = 0; j < n_groups && g < 0; ++j) {
+            const int32_t* cj = hist + g_first[j] + q;
+            int same = 1;
+            for (int t = 0; t < w; ++t)
+                if (c[t] != cj[t]) { same = 0; break; }
+            if (same) g = j;
+        }
+        if (g < 0) {
+            g = n_groups++;
+            g_first[g] = i;
+            g_count[g] = 0;
+            g_last[g] = i;
+        }
+        g_count[g] += 1;
+        if (i > g_last[g]) g_last[g] = i;
+    }
+    int n_out = 0;
+    while (n_out < topk && n_out < n_groups) {
+        int best = -1;
+        for (int j = 0; j < n_groups; ++j) {
+            if (g_taken[j]) continue;
+            if (best < 0 || g_count[j] > g_count[best] ||
+                (g_count[j] == g_count[best] && g_last[j] > g_last[best]))
+                best = j;
+        }
+        g_taken[best] = 1;
+        for (int t = 0; t < w; ++t) rows[n_out * w + t] = hist[g_last[best] + q + t];
+        if (counts) counts[n_out] = g_count[best];
+        if (lasts) lasts[n_out] = g_last[best];
+        ++n_out;
+    }
+    free(g_first); free(g_count); free(g_last); free(g_taken);
+    return n_out;
+}
+
+/* ------------------------------------------------------------------ extended model bigram (Section 4.1, "Extensions")
+ *
+ * T[V, k_tab] holds, per token x, the k_tab most likely next tokens of the model
+ * bigram in rank order.  The rank-r draft of width w after x starts with T[x][r]
+ * and continues by the top-1 bigram: s_{j+1} = T[s_j][0].
+ * ext is [V, k_tab, w].
+ */
+void oracle_extend_table(const int32_t* T, int V, int k_tab, int w, int32_t* ext) {
+    for (int x = 0; x < V; ++x)
+        for (int r = 0; r < k_tab; ++r) {
+            int32_t s = T[(long)x * k_tab + r];
+            for (int j = 0; j < w; ++j) {
+                ext[((long)x * k_tab + r) * w + j] = s;
+                s = T[(long)s * k_tab + 0];
+            }
+        }
+}
+
+/* ------------------------------------------------------------------ mixed strategy (Section 4.3)
+ *
+ * Fill the B draft rows of one sequence: context N-gram rows first, query lengths
+ * in the caller's priority order, at most topk rows each; then, if asked, the
+ * extended model bigram of the last token in rank order.  With dedup a row equal
+ * in all w tokens to one already taken is skipped.  Unused rows are -1.
+ * flags: bit0 = dedup, bit1 = model fill.
+ * src[b] = q of the strategy that produced row b, 0 for the model, -1 unused.
+ */
+int oracle_draft_sequence(const int32_t* hist, int L, const int* qs, int n_q, int topk, int B, int w,
+                          int flags, const int32_t* T, int V, int k_tab,
+                          int32_t* drafts, int32_t* src, int32_t* counts) {
+    int dedup = flags & 1, model_fill = flags & 2;
+    int n = 0;
+    for (int i = 0; i < B * w; ++i) drafts[i] = -1;
+    for (int b = 0; b < B; ++b) { src[b] = -1; counts[b] = 0; }
+    int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > k_tab ? topk : k_tab) * (size_t)w);
+    int32_t* cnt = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > 0 ? topk : 1));
+    for (int qi = 0; qi < n_q && n < B; ++qi) {
+        int m = oracle_context_draft(hist, L, qs[qi], w, topk, cand, cnt, NULL);
+        for (int r = 0; r < m && n < B; ++r) {
+            int dup = 0;
+            if (dedup)
+                for (int b = 0; b < n && !dup; ++b)
+                    if (memcmp(drafts + b * w, cand + r * w, sizeof(int32_t) * (size_t)w) == 0) dup = 1;
+            if (dup) continue;
+            memcpy(drafts + n * w, cand + r * w, sizeof(int32_t) * (size_t)w);
+            src[n] = qs[qi];
+            counts[n] = cnt[r];
+            ++n;
+        }
+    }
+    if (model_fill && T && L >= 1) {
+        int32_t x = hist[L - 1];
+        for (int r = 0; r < k_tab && n < B; ++r) {
+            int32_t s = T[(long)x * k_tab + r];
+            for (int j = 0; j < w; ++j) {
+                cand[j] = s;
+                s = T[(long)s * k_tab + 0];
+            }
+            int dup = 0;
+            if (dedup)
+                for (int b = 0; b < n && !dup; ++b)
+                    if (memcmp(drafts + b * w, cand, sizeof(int32_t) * (size_t)w) == 0) dup = 1;
+            if (dup) continue;
+            memcpy(drafts + n * w, cand, sizeof(int32_t) * (size_t)w);
+            src[n] = 0;
+            counts[n] = 0;
+            ++n;
+        }
+    }
+    free(cand); free(cnt);
+    (void)V;
+    return n;
+}
+
+/* All S sequences; hist is [S, cap]. */
+void oracle_draft_batch(const int32_t* hist, const int32_t* len, int S, int cap, const int* qs, int n_q,
+                        int topk, int B, int w, int flags, const int32_t* T, int V, int k_tab,
+                        int32_t* drafts, int32_t* n_drafts, int32_t* src, int32_t* counts) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int s = 0; s < S; ++s)
+        n_drafts[s] = oracle_draft_sequence(hist + (long)s * cap, len[s], qs, n_q, topk, B, w, flags, T, V, k_tab,
+                                            drafts + (long)s * B * w, src + (long)s * B, counts + (long)s * B);
+}
+
+/* ------------------------------------------------------------------ LM head (Sections 3 and 4.1)
+ *
+ * z[y] = sum_t A[x, t] * W[y, t], bf16 inputs, fp64 products and sums.
+ * A has its own row count; W is [V, d].  rowsel (or NULL = 0..n_rows-1) picks
+ * which rows of A are evaluated, so large problems can be sampled row by row.
+ */
+static void logits_row(const uint16_t* a, const uint16_t* W, int V, int d, double* z) {
+    for (int y = 0; y < V; ++y) {
+        const uint16_t* wy = W + (long)y * d;
+        double acc = 0.0;
+        for (int t = 0; t < d; ++t) acc += bf16_to_double(a[t]) * bf16_to_double(wy[t]);
+        z[y] = acc;
+    }
+}
+
+void oracle_logits_rows(const uint16_t* A, const int64_t* rowsel, int n_rows, const uint16_t* W, int V, int d,
+                        double* out /*[n_rows, V]*/) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        long x = rowsel ? (long)rowsel[r] : r;
+        logits_row(A + x * d, W, V, d, out + (long)r * V);
+    }
+}
+
+/* Model bigram table rows: the k largest logits of each selected row, value
+ * descending, equal values by ascending token id.  idx/val are [n_rows, k]. */
+void oracle_topk_rows(const uint16_t* A, const int64_t* rowsel, int n_rows, const uint16_t* W, int V, int d,
+                      int k, int32_t* idx, double* val) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        long x = rowsel ? (long)rowsel[r] : r;
+        double* z = (double*)malloc(sizeof(double) * (size_t)V);
+        char* used = (char*)calloc((size_t)V, 1);
+        logits_row(A + x * d, W, V, d, z);
+        for (int j = 0; j < k; ++j) {
+            int best = -1;
+            for (int y = 0; y < V; ++y)
+                if (!used[y] && (best < 0 || z[y] > z[best])) best = y; /* strict > keeps the lowest id */
+            if (best < 0) { idx[(long)r * k + j] = -1; if (val) val[(long)r * k + j] = -INFINITY; continue; }
+            used[best] = 1;
+            idx[(long)r * k + j] = best;
+            if (val) val[(long)r * k + j] = z[best];
+        }
+        free(z); free(used);
+    }
+}
+
+/* Verification: the greedy next token at each selected position, lowest id on
+ * exact ties, with the winning logit and the gap to the runner-up. */
+void oracle_verify_rows(const uint16_t* H, const int64_t* rowsel, int n_rows, const uint16_t* W, int V, int d,
+                        int32_t* argmax, double* maxval, double* gap) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        long m = rowsel ? (long)rowsel[r] : r;
+        double* z = (double*)malloc(sizeof(double) * (size_t)V);
+        logits_row(H + m * d, W, V, d, z);
+        int best = 0;
+        for (int y = 1; y < V; ++y)
+            if (z[y] > z[best]) best = y;
+        double second = -INFINITY;
+        for (int y = 0; y < V; ++y)
+            if (y != best && z[y] > second) second = z[y];
+        argmax[r] = best;
+        if (maxval) maxval[r] = z[best];
+        if (gap) gap[r] = z[best] - second;
+        free(z);
+    }
+}
+
+/* ------------------------------------------------------------------ greedy acceptance (Sections 1, 5 and Appendix D)
+ *
+ * Row b of the verify block is [x_L, s_1 .. s_w]; P[b][j] is the model's greedy
+ * token after column j.  a_b = the longest prefix with s_{j+1} == P[b][j].  The row
+ * with the longest accepted prefix wins (lowest b on ties); its a tokens and the
+ * bonus token P[b*][a] are appended to the history: a+1 tokens per call.
+ * A sequence whose history cannot take a+1 more tokens commits nothing and
+ * reports acc_len = best_row = -1.  With no drafts, row 0 / a = 0 is used.
+ * drafts [S,B,w], P [S,B,w+1], hist [S,cap], committed [S,w+1] padded with -1.
+ */
+void oracle_accept_commit(const int32_t* drafts, const int32_t* n_drafts, const int32_t* P, int S, int B, int w,
+                          int32_t* hist, int32_t* len, int cap,
+                          int32_t* acc_len, int32_t* best_row, int32_t* committed) {
+#pragma omp parallel for schedule(static)
+    for (int s = 0; s < S; ++s) {
+        const int32_t* ds = drafts + (long)s * B * w;
+        const int32_t* ps = P + (long)s * B * (w + 1);
+        int nb = n_drafts[s];
+        int best_b = 0, best_a = 0;
+        for (int b = 0; b < nb; ++b) {
+            int a = 0;
+            while (a < w && ds[b * w + a] == ps[b * (w + 1) + a]) ++a;
+            if (a > best_a) { best_a = a; best_b = b; }
+        }
+        for (int j = 0; j <= w; ++j) committed[(long)s * (w + 1) + j] = -1;
+        int L = len[s];
+        if (L + best_a + 1 > cap) {
+            acc_len[s] = -1;
+            best_row[s] = -1;
+            continue;
+        }
+        for (int j = 0; j < best_a; ++j) committed[(long)s * (w + 1) + j] = ds[best_b * w + j];
+        committed[(long)s * (w + 1) + best_a] = ps[best_b * (w + 1) + best_a];
+        for (int j = 0; j <= best_a; ++j) hist[(long)s * cap + L + j] = committed[(long)s * (w + 1) + j];
+        len[s] = L + best_a + 1;
+        acc_len[s] = best_a;
+        best_row[s] = best_b;
+    }
+}

@@ -1,0 +1,158 @@
+"""Pins for the oracle's greedy acceptance, commit, mixing and table extension."""
+import os
+
+import numpy as np
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def brute_accept(drafts, nd, P, hist, lens):
+    drafts, P, hist, lens = drafts.copy(), P.copy(), hist.copy(), lens.copy()
+    S, B, w = drafts.shape
+    cap = hist.shape[1]
+    acc, best, com = [], [], []
+    for s in range(S):
+        lengths = []
+        for b in range(int(nd[s])):
+            n = 0
+            for j in range(w):
+                if drafts[s, b, j] != P[s, b, j]:
+                    break
+                n += 1
+            lengths.append(n)
+        if lengths:
+            a = max(lengths)
+            bb = lengths.index(a)
+        else:
+            a, bb = 0, 0
+        toks = [int(t) for t in drafts[s, bb, :a]] + [int(P[s, bb, a])]
+        if lens[s] + len(toks) > cap:
+            acc.append(-1); best.append(-1); com.append([-1] * (w + 1))
+            continue
+        hist[s, lens[s]:lens[s] + len(toks)] = toks
+        lens[s] += len(toks)
+        acc.append(a); best.append(bb); com.append(toks + [-1] * (w + 1 - len(toks)))
+    return np.array(acc), np.array(best), np.array(com), hist, lens
+
+
+def test_hand_example_from_golden_file():
+    d, p, exp = [], [], {}
+    for line in open(os.path.join(GOLD, "accept_hand_example.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        key, rest = line.split(" ", 1)
+        vals = [int(t) for t in rest.split()]
+        if key == "draft":
+            d.append(vals)
+        elif key == "pred":
+            p.append(vals)
+        else:
+            exp[key] = vals
+    drafts = np.array([d], np.int32)
+    P = np.array([p], np.int32)
+    hist = np.full((1, 8), -1, np.int32)
+    hist[0, :2] = [1, 5]
+    lens = np.array([2], np.int32)
+    acc, best, com = oracle.accept_commit(drafts, np.array([3], np.int32), P, hist, lens)
+    assert acc.tolist() == [max(exp["accepted"])] and best.tolist() == exp["best"]
+    assert com[0].tolist() == exp["committed"]
+    assert hist[0].tolist() == [1, 5] + exp["committed"] + [-1] * 3 and lens.tolist() == [5]
+    # each row on its own reproduces the per-row accepted lengths
+    for b, a in enumerate(exp["accepted"]):
+        h = np.full((1, 8), -1, np.int32)
+        acc1, _, _ = oracle.accept_commit(drafts[:, b:b + 1], np.array([1], np.int32), P[:, b:b + 1], h,
+                                          np.array([0], np.int32))
+        assert acc1.tolist() == [a]
+
+
+def test_brute_force_small_alphabet():
+    g = np.random.default_rng(11)
+    for trial in range(200):
+        S, B, w = int(g.integers(1, 5)), int(g.integers(1, 7)), int(g.integers(1, 6))
+        A = int(g.integers(2, 4))
+        drafts = g.integers(0, A, (S, B, w)).astype(np.int32)
+        P = g.integers(0, A, (S, B, w + 1)).astype(np.int32)
+        nd = g.integers(0, B + 1, S).astype(np.int32)
+        cap = 12
+        lens = g.integers(0, cap + 1, S).astype(np.int32)   # some sequences cannot take the commit
+        hist = np.full((S, cap), -1, np.int32)
+        for s in range(S):
+            hist[s, :lens[s]] = g.integers(0, A, lens[s])
+        e_acc, e_best, e_com, e_hist, e_lens = brute_accept(drafts, nd, P, hist, lens)
+        acc, best, com = oracle.accept_commit(drafts, nd, P, hist, lens)
+        assert np.array_equal(acc, e_acc) and np.array_equal(best, e_best) and np.array_equal(com, e_com)
+        assert np.array_equal(hist, e_hist) and np.array_equal(lens, e_lens)
+
+
+def test_no_drafts_commits_the_plain_greedy_token():
+    drafts = np.full((1, 2, 3), -1, np.int32)
+    P = np.array([[[42, 1, 2, 3], [9, 9, 9, 9]]], np.int32)
+    hist = np.full((1, 4), -1, np.int32)
+    hist[0, 0] = 7
+    lens = np.array([1], np.int32)
+    acc, best, com = oracle.accept_commit(drafts, np.array([0], np.int32), P, hist, lens)
+    assert acc.tolist() == [0] and best.tolist() == [0] and com[0].tolist() == [42, -1, -1, -1]
+    assert hist[0].tolist() == [7, 42, -1, -1] and lens.tolist() == [2]
+
+
+# ----------------------------------------------------------------------------- mixing (Section 4.3)
+def brute_mix(hist, qs, topk, B, w, flags, T):
+    from test_oracle_context import brute_context
+    rows, src, cnt = [], [], []
+    for q in qs:
+        for c, n, _ in brute_context(hist, q, w, topk):
+            if len(rows) == B:
+                break
+            if (flags & 1) and list(c) in rows:
+                continue
+            rows.append(list(c)); src.append(q); cnt.append(n)
+    if (flags & 2) and T is not None and len(hist) > 0:
+        x = int(hist[-1])
+        for r in range(T.shape[1]):
+            if len(rows) == B:
+                break
+            chain, s = [], int(T[x, r])
+            for _ in range(w):
+                chain.append(s)
+                s = int(T[s, 0])
+            if (flags & 1) and chain in rows:
+                continue
+            rows.append(chain); src.append(0); cnt.append(0)
+    return rows, src, cnt
+
+
+def test_mixing_against_brute_force():
+    g = np.random.default_rng(5)
+    V, k_tab = 5, 3
+    for trial in range(300):
+        T = np.stack([g.permutation(V)[:k_tab] for _ in range(V)]).astype(np.int32)
+        L = int(g.integers(0, 60))
+        hist = g.integers(0, V, L).astype(np.int32)
+        n_q = int(g.integers(0, 4))
+        qs = [int(q) for q in g.permutation([1, 2, 3, 4])[:n_q]]
+        topk, B, w = int(g.integers(1, 5)), int(g.integers(1, 9)), int(g.integers(1, 5))
+        flags = int(g.integers(0, 4))
+        cap = (L + 3) // 4 * 4 + 4
+        h2 = np.full((1, cap), -1, np.int32)
+        h2[0, :L] = hist
+        drafts, nd, src, cnt = oracle.draft_batch(h2, np.array([L], np.int32), qs, topk, B, w, flags, T)
+        rows, esrc, ecnt = brute_mix(hist, qs, topk, B, w, flags, T)
+        n = len(rows)
+        assert nd[0] == n
+        assert drafts[0, :n].tolist() == rows and (drafts[0, n:] == -1).all()
+        assert src[0, :n].tolist() == esrc and (src[0, n:] == -1).all()
+        assert cnt[0, :n].tolist() == ecnt and (cnt[0, n:] == 0).all()
+
+
+def test_context_rows_come_first_then_model_rows_in_rank_order():
+    T = np.array([[1, 2, 0], [2, 0, 1], [0, 1, 2]], np.int32)   # top-1 chain 0->1->2->0
+    hist = np.array([[0, 1, 2, 0, 1, 2, 0, -1]], np.int32)
+    drafts, nd, src, cnt = oracle.draft_batch(hist, np.array([7], np.int32), [1], 2, 4, 2, 3, T)
+    # context after token 0: (1,2) seen twice; model ranks: (1,2) duplicate dropped, (2,0), (0,1)
+    assert nd[0] == 3 and drafts[0].tolist() == [[1, 2], [2, 0], [0, 1], [-1, -1]]
+    assert src[0].tolist() == [1, 0, 0, -1] and cnt[0].tolist() == [2, 0, 0, 0]
+    drafts, nd, src, _ = oracle.draft_batch(hist, np.array([7], np.int32), [1], 2, 4, 2, 2, T)  # no dedup
+    assert nd[0] == 4 and drafts[0].tolist() == [[1, 2], [1, 2], [2, 0], [0, 1]]

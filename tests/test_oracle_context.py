@@ -1,0 +1,118 @@
+"""Pins for the oracle's context N-gram (Section 4.2) against things other than itself."""
+import collections
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def brute_context(hist, q, w, topk):
+    """Independent restatement with a dict keyed by the continuation tuple."""
+    hist = list(int(t) for t in hist)
+    L = len(hist)
+    if L < q + w:
+        return []
+    query = tuple(hist[L - q:])
+    groups = {}
+    for i in range(0, L - q - w + 1):
+        if tuple(hist[i:i + q]) == query:
+            c = tuple(hist[i + q:i + q + w])
+            cnt, last = groups.get(c, (0, -1))
+            groups[c] = (cnt + 1, max(last, i))
+    order = sorted(groups.items(), key=lambda kv: (-kv[1][0], -kv[1][1]))
+    return [(c, cnt, last) for c, (cnt, last) in order[:topk]]
+
+
+def as_list(res):
+    rows, counts, lasts = res
+    return [(tuple(int(t) for t in r), int(c), int(l)) for r, c, l in zip(rows, counts, lasts)]
+
+
+def test_hand_example_from_golden_file():
+    hist = q = w = None
+    rows = []
+    for line in open(os.path.join(GOLD, "context_hand_example.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        key, rest = line.split(" ", 1)
+        if key == "hist":
+            hist = [int(t) for t in rest.split()]
+        elif key == "q":
+            q = int(rest)
+        elif key == "w":
+            w = int(rest)
+        elif key == "row":
+            toks, cnt, last = rest.split("|")
+            rows.append((tuple(int(t) for t in toks.split()), int(cnt), int(last)))
+    assert as_list(oracle.context_draft(hist, q, w, 3)) == rows
+    assert as_list(oracle.context_draft(hist, q, w, 2)) == rows[:2]
+    assert as_list(oracle.context_draft(hist, q, w, 8)) == rows
+
+
+@pytest.mark.parametrize("vocab", [2, 3, 4])
+def test_brute_force_on_tiny_histories_with_many_ties(vocab):
+    g = np.random.default_rng(100 + vocab)
+    for trial in range(300):
+        L = int(g.integers(0, 65))
+        q = int(g.integers(1, 5))
+        w = int(g.integers(1, 5))
+        topk = int(g.integers(1, 9))
+        hist = g.integers(0, vocab, L).astype(np.int32)
+        assert as_list(oracle.context_draft(hist, q, w, topk)) == brute_context(hist, q, w, topk), (L, q, w, topk)
+
+
+def test_library_unique_gives_the_same_groups_and_counts():
+    # numpy's sliding windows + unique(axis=0) restate "count each distinct (q+w)-gram
+    # whose first q tokens equal the query" with library routines.
+    g = np.random.default_rng(7)
+    for trial in range(50):
+        L, q, w = int(g.integers(8, 400)), int(g.integers(1, 4)), int(g.integers(1, 6))
+        hist = g.integers(0, 6, L).astype(np.int32)
+        win = np.lib.stride_tricks.sliding_window_view(hist, q + w)
+        m = win[(win[:, :q] == hist[L - q:]).all(axis=1)]
+        rows, counts, _ = oracle.context_draft(hist, q, w, topk=10 ** 6)
+        if len(m) == 0:
+            assert len(rows) == 0
+            continue
+        u, c = np.unique(m[:, q:], axis=0, return_counts=True)
+        want = collections.Counter({tuple(r): int(n) for r, n in zip(u.tolist(), c.tolist())})
+        got = collections.Counter({tuple(r): int(n) for r, n in zip(rows.tolist(), counts.tolist())})
+        assert got == want
+        assert sum(got.values()) == len(m)
+
+
+def test_invariants():
+    # constant history: one group holding every eligible window
+    L, q, w = 50, 2, 3
+    rows, counts, lasts = oracle.context_draft(np.full(L, 9, np.int32), q, w, 4)
+    assert rows.tolist() == [[9, 9, 9]] and counts.tolist() == [L - q - w + 1] and lasts.tolist() == [L - q - w]
+    # q = w = 1 is the next-token histogram of the last token (excluding the final position)
+    g = np.random.default_rng(3)
+    hist = g.integers(0, 5, 200).astype(np.int32)
+    nxt = collections.Counter(int(hist[i + 1]) for i in range(len(hist) - 1) if hist[i] == hist[-1])
+    rows, counts, _ = oracle.context_draft(hist, 1, 1, 100)
+    assert {int(r[0]): int(c) for r, c in zip(rows, counts)} == dict(nxt)
+    assert all(counts[i] >= counts[i + 1] for i in range(len(counts) - 1))
+    # relabelling the vocabulary relabels the output and nothing else
+    perm = g.permutation(5).astype(np.int32)
+    r2, c2, l2 = oracle.context_draft(perm[hist], 1, 1, 100)
+    assert np.array_equal(r2, perm[rows]) and np.array_equal(c2, counts)
+    # too short for one full window -> nothing
+    assert len(oracle.context_draft(np.array([1, 1, 1], np.int32), 2, 2, 4)[0]) == 0
+    assert len(oracle.context_draft(np.array([], np.int32), 1, 1, 4)[0]) == 0
+    # exactly one full window
+    r, c, l = oracle.context_draft(np.array([1, 2, 3, 1], np.int32), 1, 2, 4)
+    assert r.tolist() == [[2, 3]] and c.tolist() == [1] and l.tolist() == [0]
+
+
+def test_later_occurrence_wins_ties_and_count_wins_over_recency():
+    #            0  1  2  3  4  5  6  7  8  9 10
+    hist = [4, 1, 4, 2, 4, 1, 4, 3, 4, 2, 4]
+    rows, counts, lasts = oracle.context_draft(np.array(hist, np.int32), 1, 1, 3)
+    # after 4: 1 (x2, last 4), 2 (x2, last 8), 3 (x1, last 6); window 10 has no continuation
+    assert rows.reshape(-1).tolist() == [2, 1, 3] and counts.tolist() == [2, 2, 1] and lasts.tolist() == [8, 4, 6]
