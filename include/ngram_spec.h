@@ -1,0 +1,158 @@
+/*
+ * ngram_spec.h -- C ABI of the batched N-gram speculation step for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel part of learning-free batched speculative
+ * decoding ("The N-Grammys", arXiv 2411.03786):
+ *
+ *   draft_context_ngrams      context N-gram drafts + mixed allocation   (Sections 4.2, 4.3)
+ *   build_model_ngram_tables  model bigram table and its w-token extension (Section 4.1)
+ *   verify_lmhead_argmax      LM-head part of the batched verification call (Sections 3, 4.1)
+ *   accept_and_commit         greedy acceptance, best row, history update  (Sections 1, 5, App. D)
+ *
+ * Conventions
+ *   - Every function returns 0 (SPEC_OK) or a negative SPEC_ERR_* code; nothing throws or aborts.
+ *     After an error spec_last_error() gives a one-line reason.
+ *   - Pointers named d_* are DEVICE pointers owned by the caller, 16-byte aligned, and must stay
+ *     valid until the stream work that uses them has finished.  Other pointers are host pointers.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All calls are
+ *     asynchronous with respect to the host except spec_init, spec_destroy and spec_get_status.
+ *   - Tokens are int32 in [0, V).  A history matrix is hist[S, cap] (row stride cap, cap % 4 == 0)
+ *     with len[S] valid tokens per row.
+ *   - Symbols: S sequences, B draft rows per sequence, w drafted tokens per row, q = number of
+ *     trailing context tokens matched (an "N-gram" has q = N-1), V vocabulary size, d hidden
+ *     size, k_tab = entries kept per row of the model bigram table, M = S*B*(w+1) verify rows.
+ *   - Limits: 1 <= B <= 64, 1 <= w <= 16, 1 <= q <= 4, n_q <= 4, 1 <= topk <= B, 1 <= k_tab <= 32,
+ *     d % 8 == 0, M <= SPEC_MAX_VERIFY_ROWS, history length < 2^28.
+ *   - Data errors found on the device (token out of range, history overflow, a bounded wait that
+ *     expired) never trap: they set bits in a status word that spec_get_status returns.
+ *   - The GPU must be compute capability 10.0 (sm_100a).  There is no CPU fallback: every entry
+ *     point fails with SPEC_ERR_CUDA when no such device is usable.
+ */
+#ifndef NGRAM_SPEC_H_
+#define NGRAM_SPEC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct spec_ctx spec_ctx;
+
+enum {
+    SPEC_OK = 0,
+    SPEC_ERR_ARG = -1,         /* null / misaligned pointer, size out of the documented limits */
+    SPEC_ERR_UNSUPPORTED = -2, /* valid request the library does not implement */
+    SPEC_ERR_CUDA = -3,        /* a CUDA runtime / driver call failed, or no sm_100 device */
+    SPEC_ERR_NOT_BUILT = -4    /* model fill requested before build_model_ngram_tables */
+};
+
+/* bits of the device status word */
+enum {
+    SPEC_STATUS_TOKEN_RANGE = 1, /* a token outside [0, V) was met; the affected row was dropped */
+    SPEC_STATUS_CAPACITY = 2,    /* len > cap, or a commit did not fit: that sequence was skipped */
+    SPEC_STATUS_TIMEOUT = 4,     /* a bounded device-side wait expired; results of that call are invalid */
+    SPEC_STATUS_GROUPS = 8       /* more distinct continuations than the drafter can group exactly */
+};
+
+enum { SPEC_F32 = 0, SPEC_BF16 = 1 };
+enum { SPEC_FLAG_DEDUP = 1, SPEC_FLAG_MODEL_FILL = 2 };
+enum { SPEC_MAX_VERIFY_ROWS = 65536 };
+
+/*
+ * Create a context for one model head on one device.
+ *   d_embed    [V, d] input embedding matrix (the paper's V, Section 4.1), row-major.
+ *   d_unembed  [V, d] output embedding = lm_head weight (the paper's U^T), row-major.
+ *   dtype      SPEC_BF16: both matrices are bfloat16 and are BORROWED (not copied; keep them alive).
+ *              SPEC_F32 : both are float32; the context OWNS a bfloat16 copy rounded once,
+ *                         round-to-nearest-even, which is what every contraction then reads.
+ *   device     CUDA device ordinal; `stream` orders the conversion copy.
+ * Allocates the context's scratch (verify merge keys, status word).  Synchronises the stream.
+ */
+int spec_init(spec_ctx** out, const void* d_embed, const void* d_unembed, int dtype, int V, int d, int device,
+              void* stream);
+
+/* Frees everything the context owns.  The caller must have finished all stream work first. */
+int spec_destroy(spec_ctx* ctx);
+
+/* Synchronises `stream`, returns the accumulated SPEC_STATUS_* bits in *status_bits and clears them. */
+int spec_get_status(spec_ctx* ctx, int* status_bits, void* stream);
+
+/* One-line description of the last error returned for this context (ctx may be NULL: global). */
+const char* spec_last_error(spec_ctx* ctx);
+
+/*
+ * Model bigram table (Section 4.1 "Bigram", "Batched drafts", "Extensions").
+ * For every token x: the k_tab largest entries of row x of Z = A * unembed^T, value descending,
+ * equal values by ascending token id.  A = d_rows if given ([V, d] bfloat16: the model's final
+ * hidden state after each single-token context), else the context's embedding matrix.
+ * bf16 x bf16 products accumulate in fp32 on the tensor cores; Z is never written to memory.
+ *   d_tab_idx  [V, k_tab] int32 out (required).  The context remembers this pointer (and d_ext)
+ *              for draft_context_ngrams; keep it alive.
+ *   d_tab_val  [V, k_tab] float32 out or NULL.
+ *   d_ext      [V, k_tab, w_ext] int32 out or NULL: ext[x][r][0] = T[x][r], ext[x][r][j+1] =
+ *              T[ext[x][r][j]][0] (rank-r first token, then top-1 chaining).  w_ext = 0 => none.
+ * Allocates (and keeps) scratch for partial top-k lists on first use; asynchronous afterwards.
+ */
+int build_model_ngram_tables(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx,
+                             float* d_tab_val, int32_t* d_ext, void* stream);
+
+/* Adopt a table built earlier (e.g. loaded from disk) instead of building it. */
+int spec_set_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, const int32_t* d_ext, int w_ext);
+
+/*
+ * Drafting (Sections 4.2 and 4.3).  Per sequence and per q in qs (caller's priority order): every
+ * earlier full window of q+w tokens whose first q tokens equal the last q tokens of the history
+ * is a match; matches are grouped by their w-token continuation; groups are ranked by count
+ * descending, ties by the later occurrence; the first topk continuations become draft rows.
+ * Rows are taken in qs order; with SPEC_FLAG_DEDUP a row equal to an earlier row is skipped; with
+ * SPEC_FLAG_MODEL_FILL the remaining rows are the extended model bigram of the last token in rank
+ * order.  Histories shorter than q+w give no rows for that q.
+ *   qs         host array of n_q query lengths (n_q = 0: model rows only).
+ *   d_drafts   [S, B, w] out, unused rows = -1.      d_ndrafts [S] out.
+ *   d_src      [S, B] out or NULL: q of the producing strategy, 0 = model, -1 = unused.
+ *   d_counts   [S, B] out or NULL: occurrence count of a context row, 0 otherwise.
+ */
+int draft_context_ngrams(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap,
+                         const int* qs, int n_q, int topk, int B, int w, int flags, int32_t* d_drafts,
+                         int32_t* d_ndrafts, int32_t* d_src, int32_t* d_counts, void* stream);
+
+/*
+ * Verification head (Section 3: the model call on a (k, w+1) block; here its LM-head part).
+ * d_argmax[m] = argmax_y <hidden[m, :], unembed[y, :]>, lowest y on exact ties; the [M, V] logits
+ * are never written.  Row m = (s*B + b)*(w+1) + j holds the hidden state at column j of draft row
+ * b of sequence s (column 0 = the last context token).
+ *   d_hidden   [M, d] bfloat16.      d_max  [M] float32 out or NULL (the winning logit).
+ * Uses the context's merge keys as scratch: calls on one context must not overlap on the GPU.
+ */
+int verify_lmhead_argmax(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max,
+                         void* stream);
+
+/*
+ * Greedy acceptance and commit (Section 1: accept what the model would have predicted;
+ * Appendix D: keep the row with the longest accepted speculation; Section 5: tokens per call).
+ * a_b = longest prefix of draft row b with drafts[b][j] == argmax[b][j]; best row = largest a_b,
+ * lowest b on ties (row 0, a = 0 when the sequence has no drafts).  Appends the a accepted tokens
+ * and the bonus token argmax[b*][a] to the history and adds a+1 to len.  A sequence whose history
+ * cannot take a+1 more tokens is left untouched, reports acc_len = best_row = -1 and sets
+ * SPEC_STATUS_CAPACITY.
+ *   d_argmax    [S, B, w+1] from verify_lmhead_argmax.
+ *   d_acc_len   [S] out.   d_best_row [S] out.   d_committed [S, w+1] out, padded with -1.
+ */
+int accept_and_commit(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_ndrafts, const int32_t* d_argmax,
+                      int S, int B, int w, int32_t* d_hist, int32_t* d_len, int cap, int32_t* d_acc_len,
+                      int32_t* d_best_row, int32_t* d_committed, void* stream);
+
+/*
+ * Test aid: the same tensor-core main loop as the two head calls with a plain store epilogue.
+ * d_logits[i, y] = <rows[i, :], unembed[y, :]> for i < m, as float32 [m, V].
+ */
+int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, void* stream);
+
+/* Number of kernels the library has launched for this context since spec_init. */
+long long spec_launch_count(spec_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NGRAM_SPEC_H_ */

@@ -1,0 +1,238 @@
+// Host side of the C ABI: context life cycle, argument checks, error strings.
+#include <stdarg.h>
+#include <string.h>
+
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+static char g_err[256] = "";
+
+namespace ngs {
+
+int fail(spec_ctx* ctx, int code, const char* fmt, ...) {
+    char buf[256];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    strncpy(ctx ? ctx->err : g_err, buf, 255);
+    return code;
+}
+
+int check_cuda(spec_ctx* ctx, cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return SPEC_OK;
+    return fail(ctx, SPEC_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ctx, SPEC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return SPEC_OK;
+}
+
+__global__ void round_f32_to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
+}
+
+}  // namespace ngs
+
+using namespace ngs;
+
+extern "C" {
+
+const char* spec_last_error(spec_ctx* ctx) { return ctx ? ctx->err : g_err; }
+
+long long spec_launch_count(spec_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int spec_init(spec_ctx** out, const void* d_embed, const void* d_unembed, int dtype, int V, int d, int device,
+              void* stream) {
+    if (!out) return fail(nullptr, SPEC_ERR_ARG, "spec_init: out is NULL");
+    *out = nullptr;
+    if (!d_embed || !d_unembed) return fail(nullptr, SPEC_ERR_ARG, "spec_init: weight pointer is NULL");
+    if (!aligned16(d_embed) || !aligned16(d_unembed))
+        return fail(nullptr, SPEC_ERR_ARG, "spec_init: weight pointers must be 16-byte aligned");
+    if (V <= 0 || d <= 0 || d % 8 != 0) return fail(nullptr, SPEC_ERR_ARG, "spec_init: need V > 0, d > 0, d %% 8 == 0");
+    if (dtype != SPEC_F32 && dtype != SPEC_BF16) return fail(nullptr, SPEC_ERR_ARG, "spec_init: unknown dtype %d", dtype);
+    int n_dev = 0;
+    cudaError_t e = cudaGetDeviceCount(&n_dev);
+    if (e != cudaSuccess || n_dev <= 0)
+        return fail(nullptr, SPEC_ERR_CUDA, "spec_init: no CUDA device (%s); this library has no CPU path",
+                    cudaGetErrorString(e));
+    if (device < 0 || device >= n_dev) return fail(nullptr, SPEC_ERR_ARG, "spec_init: device %d out of range", device);
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, device)) != cudaSuccess) return check_cuda(nullptr, e, "cudaGetDeviceProperties");
+    if (prop.major != 10)
+        return fail(nullptr, SPEC_ERR_CUDA, "spec_init: device %d is sm_%d%d; the kernels are built for sm_100a only",
+                    device, prop.major, prop.minor);
+    if ((e = cudaSetDevice(device)) != cudaSuccess) return check_cuda(nullptr, e, "cudaSetDevice");
+
+    spec_ctx* ctx = new spec_ctx();
+    ctx->device = device;
+    ctx->V = V;
+    ctx->d = d;
+    ctx->num_sms = prop.multiProcessorCount;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = SPEC_OK;
+    do {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) {
+            rc = fail(nullptr, SPEC_ERR_CUDA, "spec_init: cuTensorMapEncodeTiled not available from the driver");
+            break;
+        }
+        ctx->encode = (EncodeTiledFn)fn;
+        if (dtype == SPEC_F32) {
+            size_t n = (size_t)V * d;
+            if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->owned_embed, n * 2), "cudaMalloc(embed)"))) break;
+            if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->owned_unembed, n * 2), "cudaMalloc(unembed)"))) break;
+            int blocks = ctx->num_sms * 8;
+            round_f32_to_bf16_kernel<<<blocks, 256, 0, st>>>((const float*)d_embed, (__nv_bfloat16*)ctx->owned_embed, n);
+            round_f32_to_bf16_kernel<<<blocks, 256, 0, st>>>((const float*)d_unembed, (__nv_bfloat16*)ctx->owned_unembed, n);
+            ctx->launches += 2;
+            ctx->embed = ctx->owned_embed;
+            ctx->unembed = ctx->owned_unembed;
+        } else {
+            ctx->embed = d_embed;
+            ctx->unembed = d_unembed;
+        }
+        if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_status, sizeof(int)), "cudaMalloc(status)"))) break;
+        if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_keys, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS),
+                             "cudaMalloc(keys)"))) break;
+        if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_ticket, sizeof(unsigned int)), "cudaMalloc(ticket)"))) break;
+        cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st);
+        cudaMemsetAsync(ctx->d_keys, 0, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS, st);
+        cudaMemsetAsync(ctx->d_ticket, 0, sizeof(unsigned int), st);
+        if ((rc = make_tensor_map(ctx, &ctx->tm_unembed, ctx->unembed, V, d, 32))) {
+            strncpy(g_err, ctx->err, 255);
+            break;
+        }
+        if ((rc = check_cuda(nullptr, cudaStreamSynchronize(st), "spec_init: stream sync"))) break;
+    } while (0);
+    if (rc != SPEC_OK) {
+        spec_destroy(ctx);
+        return rc;
+    }
+    *out = ctx;
+    return SPEC_OK;
+}
+
+int spec_destroy(spec_ctx* ctx) {
+    if (!ctx) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->owned_embed);
+    cudaFree(ctx->owned_unembed);
+    cudaFree(ctx->d_status);
+    cudaFree(ctx->d_keys);
+    cudaFree(ctx->d_ticket);
+    cudaFree(ctx->d_part_val);
+    cudaFree(ctx->d_part_idx);
+    delete ctx;
+    return SPEC_OK;
+}
+
+int spec_get_status(spec_ctx* ctx, int* status_bits, void* stream) {
+    if (!ctx || !status_bits) return fail(ctx, SPEC_ERR_ARG, "spec_get_status: NULL argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = check_cuda(ctx, cudaMemcpyAsync(status_bits, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st),
+                        "spec_get_status: copy");
+    if (rc) return rc;
+    if ((rc = check_cuda(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st), "spec_get_status: clear"))) return rc;
+    return check_cuda(ctx, cudaStreamSynchronize(st), "spec_get_status: sync");
+}
+
+int spec_set_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, const int32_t* d_ext, int w_ext) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_set_model_table: ctx is NULL");
+    if (!d_tab_idx || k_tab < 1 || k_tab > kMaxKTab) return fail(ctx, SPEC_ERR_ARG, "spec_set_model_table: bad table");
+    if (d_ext && (w_ext < 1 || w_ext > kMaxW)) return fail(ctx, SPEC_ERR_ARG, "spec_set_model_table: bad w_ext");
+    ctx->tab_idx = d_tab_idx;
+    ctx->k_tab = k_tab;
+    ctx->ext = d_ext;
+    ctx->w_ext = d_ext ? w_ext : 0;
+    return SPEC_OK;
+}
+
+int build_model_ngram_tables(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx,
+                             float* d_tab_val, int32_t* d_ext, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "build_model_ngram_tables: ctx is NULL");
+    if (!d_tab_idx) return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_tables: d_tab_idx is NULL");
+    if (k_tab < 1 || k_tab > kMaxKTab || k_tab > ctx->V)
+        return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_tables: k_tab must be in [1, min(%d, V)]", kMaxKTab);
+    if (w_ext < 0 || w_ext > kMaxW) return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_tables: w_ext must be in [0, %d]", kMaxW);
+    if ((d_ext != nullptr) != (w_ext > 0))
+        return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_tables: d_ext and w_ext must be given together");
+    if ((d_rows && !aligned16(d_rows)) || !aligned16(d_tab_idx))
+        return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_tables: pointers must be 16-byte aligned");
+    cudaSetDevice(ctx->device);
+    int rc = launch_table(ctx, d_rows ? d_rows : ctx->embed, k_tab, w_ext, d_tab_idx, d_tab_val, d_ext,
+                          (cudaStream_t)stream);
+    if (rc) return rc;
+    return spec_set_model_table(ctx, d_tab_idx, k_tab, d_ext, w_ext);
+}
+
+int draft_context_ngrams(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs,
+                         int n_q, int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts,
+                         int32_t* d_src, int32_t* d_counts, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "draft_context_ngrams: ctx is NULL");
+    if (!d_hist || !d_len || !d_drafts || !d_ndrafts) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams: NULL pointer");
+    if (!aligned16(d_hist)) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams: d_hist must be 16-byte aligned");
+    if (S < 0 || cap <= 0 || cap % 4 != 0 || cap >= (1 << 28))
+        return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams: need S >= 0, 0 < cap < 2^28, cap %% 4 == 0");
+    if (B < 1 || B > kMaxB || w < 1 || w > kMaxW) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams: need 1<=B<=%d, 1<=w<=%d", kMaxB, kMaxW);
+    if (n_q < 0 || n_q > kMaxNQ || (n_q > 0 && !qs)) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams: need 0<=n_q<=%d", kMaxNQ);
+    for (int i = 0; i < n_q; ++i)
+        if (qs[i] < 1 || qs[i] > kMaxQ) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams: q must be in [1, %d]", kMaxQ);
+    if (topk < 1 || topk > B) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams: need 1 <= topk <= B");
+    if ((flags & SPEC_FLAG_MODEL_FILL) && !ctx->tab_idx)
+        return fail(ctx, SPEC_ERR_NOT_BUILT, "draft_context_ngrams: model fill needs build_model_ngram_tables first");
+    if (S == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    return launch_draft(ctx, d_hist, d_len, S, cap, qs, n_q, topk, B, w, flags, d_drafts, d_ndrafts, d_src, d_counts,
+                        (cudaStream_t)stream);
+}
+
+int verify_lmhead_argmax(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax: ctx is NULL");
+    if (!d_hidden || !d_argmax) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax: NULL pointer");
+    if (!aligned16(d_hidden)) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax: d_hidden must be 16-byte aligned");
+    if (M < 0 || M > SPEC_MAX_VERIFY_ROWS) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax: need 0 <= M <= %d", SPEC_MAX_VERIFY_ROWS);
+    if (M == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    return launch_verify(ctx, d_hidden, M, d_argmax, d_max, (cudaStream_t)stream);
+}
+
+int accept_and_commit(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_ndrafts, const int32_t* d_argmax, int S,
+                      int B, int w, int32_t* d_hist, int32_t* d_len, int cap, int32_t* d_acc_len, int32_t* d_best_row,
+                      int32_t* d_committed, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "accept_and_commit: ctx is NULL");
+    if (!d_drafts || !d_ndrafts || !d_argmax || !d_hist || !d_len || !d_acc_len || !d_best_row || !d_committed)
+        return fail(ctx, SPEC_ERR_ARG, "accept_and_commit: NULL pointer");
+    if (S < 0 || cap <= 0) return fail(ctx, SPEC_ERR_ARG, "accept_and_commit: need S >= 0, cap > 0");
+    if (B < 1 || B > kMaxB || w < 1 || w > kMaxW) return fail(ctx, SPEC_ERR_ARG, "accept_and_commit: need 1<=B<=%d, 1<=w<=%d", kMaxB, kMaxW);
+    if (S == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    return launch_accept(ctx, d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row,
+                         d_committed, (cudaStream_t)stream);
+}
+
+int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_debug_logits: ctx is NULL");
+    if (!d_rows || !d_logits || m < 0) return fail(ctx, SPEC_ERR_ARG, "spec_debug_logits: bad argument");
+    if (!aligned16(d_rows)) return fail(ctx, SPEC_ERR_ARG, "spec_debug_logits: d_rows must be 16-byte aligned");
+    if (m == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    return launch_logits(ctx, d_rows, m, d_logits, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,73 @@
+// Shared declarations of the N-gram speculation library (host side + small device helpers).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "../../include/ngram_spec.h"
+
+namespace ngs {
+
+constexpr int kMaxB = 64;
+constexpr int kMaxW = 16;
+constexpr int kMaxQ = 4;
+constexpr int kMaxNQ = 4;
+constexpr int kMaxKTab = 32;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace ngs
+
+struct spec_ctx {
+    int device = 0;
+    int V = 0, d = 0;
+    int num_sms = 0;
+    const void* embed = nullptr;    // bf16 [V, d]
+    const void* unembed = nullptr;  // bf16 [V, d]
+    void* owned_embed = nullptr;    // set when converted from fp32
+    void* owned_unembed = nullptr;
+    int* d_status = nullptr;        // device status word
+    // verify merge scratch: one packed (value, ~index) key per row + completion ticket
+    unsigned long long* d_keys = nullptr;
+    unsigned int* d_ticket = nullptr;
+    // table-build scratch: partial top-k lists per vocabulary chunk
+    float* d_part_val = nullptr;
+    int32_t* d_part_idx = nullptr;
+    size_t part_capacity = 0;  // entries
+    // model table remembered for drafting
+    const int32_t* tab_idx = nullptr;
+    int k_tab = 0;
+    const int32_t* ext = nullptr;
+    int w_ext = 0;
+    ngs::EncodeTiledFn encode = nullptr;
+    CUtensorMap tm_unembed;  // B operand of every contraction
+    long long launches = 0;
+    char err[256] = {0};
+};
+
+namespace ngs {
+
+int fail(spec_ctx* ctx, int code, const char* fmt, ...);
+int check_cuda(spec_ctx* ctx, cudaError_t e, const char* what);
+bool aligned16(const void* p);
+
+// 2-D bf16 row-major [rows, cols] tensor map, 128-byte swizzle, box = [box_rows, 64 elements].
+int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows);
+
+// head_gemm.cu
+int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st);
+int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
+                 int32_t* d_ext, cudaStream_t st);
+int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st);
+// draft.cu / accept.cu
+int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
+                 int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,
+                 int32_t* d_counts, cudaStream_t st);
+int launch_accept(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_ndrafts, const int32_t* d_argmax, int S,
+                  int B, int w, int32_t* d_hist, int32_t* d_len, int cap, int32_t* d_acc_len, int32_t* d_best_row,
+                  int32_t* d_committed, cudaStream_t st);
+
+}  // namespace ngs
