@@ -1,0 +1,12 @@
+"""B200-native batched N-gram speculation step (arXiv 2411.03786): Python binding of the C ABI.
+
+Every step runs in the CUDA library ``libngram_spec.so`` (hand-written sm_100a kernels).  This
+package only marshals arguments: torch tensors supply device memory and the stream.  There is
+no CPU path; importing works without a GPU (so the build can be checked), but creating a
+``SpecContext`` without an sm_100 device raises.
+"""
+from .binding import (FLAG_DEDUP, FLAG_MODEL_FILL, STATUS_CAPACITY, STATUS_GROUPS, STATUS_TIMEOUT,
+                      STATUS_TOKEN_RANGE, SpecContext, SpecError, declared_symbols, load_library)
+
+__all__ = ["SpecContext", "SpecError", "load_library", "declared_symbols", "FLAG_DEDUP", "FLAG_MODEL_FILL",
+           "STATUS_TOKEN_RANGE", "STATUS_CAPACITY", "STATUS_TIMEOUT", "STATUS_GROUPS"]

@@ -1,0 +1,175 @@
+"""ctypes binding of ``include/ngram_spec.h``: same names, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import re
+
+import torch
+
+from .build import LIB, build_library
+
+FLAG_DEDUP, FLAG_MODEL_FILL = 1, 2
+STATUS_TOKEN_RANGE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_GROUPS = 1, 2, 4, 8
+SPEC_F32, SPEC_BF16 = 0, 1
+
+_HEADER = os.path.join(os.path.dirname(os.path.abspath(__file__)), "..", "include", "ngram_spec.h")
+_lib = None
+
+
+class SpecError(RuntimeError):
+    pass
+
+
+def declared_symbols() -> list[str]:
+    """Function names declared in the public header."""
+    text = re.sub(r"/\*.*?\*/", "", open(_HEADER).read(), flags=re.S)
+    return sorted(set(re.findall(r"\b([a-z_][a-z0-9_]*)\s*\(", text)) - {"defined"})
+
+
+def load_library(build: bool = True) -> C.CDLL:
+    """Load (building first if needed) the CUDA library.  Fails loudly if it cannot be loaded."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build:
+        build_library()
+    if not os.path.exists(LIB):
+        raise SpecError(f"{LIB} is missing: build it with `python -m paper_2411_03786_b200.build`")
+    lib = C.CDLL(LIB)
+    vp, ip, i32p, fp = C.c_void_p, C.POINTER(C.c_int), C.c_void_p, C.c_void_p
+    lib.spec_init.argtypes = [C.POINTER(vp), vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp]
+    lib.spec_destroy.argtypes = [vp]
+    lib.spec_get_status.argtypes = [vp, ip, vp]
+    lib.spec_last_error.argtypes = [vp]
+    lib.spec_last_error.restype = C.c_char_p
+    lib.build_model_ngram_tables.argtypes = [vp, vp, C.c_int, C.c_int, i32p, fp, i32p, vp]
+    lib.spec_set_model_table.argtypes = [vp, i32p, C.c_int, i32p, C.c_int]
+    lib.draft_context_ngrams.argtypes = [vp, i32p, i32p, C.c_int, C.c_int, ip, C.c_int, C.c_int, C.c_int, C.c_int,
+                                         C.c_int, i32p, i32p, i32p, i32p, vp]
+    lib.verify_lmhead_argmax.argtypes = [vp, vp, C.c_int, i32p, fp, vp]
+    lib.accept_and_commit.argtypes = [vp, i32p, i32p, i32p, C.c_int, C.c_int, C.c_int, i32p, i32p, C.c_int, i32p,
+                                      i32p, i32p, vp]
+    lib.spec_debug_logits.argtypes = [vp, vp, C.c_int, fp, vp]
+    lib.spec_launch_count.argtypes = [vp]
+    lib.spec_launch_count.restype = C.c_longlong
+    _lib = lib
+    return lib
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, f"expected {dtype}, got {t.dtype}"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class SpecContext:
+    """One model head on one GPU.  Methods mirror the C entry points and launch on torch's current stream."""
+
+    def __init__(self, embed: torch.Tensor, unembed: torch.Tensor):
+        self._lib = load_library()
+        self._h = C.c_void_p()
+        if not torch.cuda.is_available():
+            raise SpecError("no CUDA device: this library has no CPU path")
+        assert embed.shape == unembed.shape and embed.dtype == unembed.dtype
+        dtype = {torch.float32: SPEC_F32, torch.bfloat16: SPEC_BF16}[embed.dtype]
+        self.V, self.d = int(embed.shape[0]), int(embed.shape[1])
+        self._keep = [embed, unembed]
+        rc = self._lib.spec_init(C.byref(self._h), _ptr(embed), _ptr(unembed), dtype, self.V, self.d,
+                                 embed.device.index or 0, _stream())
+        if rc != 0:
+            raise SpecError(f"spec_init failed ({rc}): {self._lib.spec_last_error(None).decode()}")
+
+    def _check(self, rc: int, what: str):
+        if rc != 0:
+            raise SpecError(f"{what} failed ({rc}): {self._lib.spec_last_error(self._h).decode()}")
+
+    def close(self):
+        if self._h:
+            torch.cuda.synchronize()
+            self._lib.spec_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def get_status(self) -> int:
+        bits = C.c_int(0)
+        self._check(self._lib.spec_get_status(self._h, C.byref(bits), _stream()), "spec_get_status")
+        return bits.value
+
+    def launch_count(self) -> int:
+        return int(self._lib.spec_launch_count(self._h))
+
+    def build_model_ngram_tables(self, k_tab: int, rows: torch.Tensor | None = None, w_ext: int = 0,
+                                 with_values: bool = False):
+        dev = self._keep[0].device
+        tab = torch.empty((self.V, k_tab), dtype=torch.int32, device=dev)
+        val = torch.empty((self.V, k_tab), dtype=torch.float32, device=dev) if with_values else None
+        ext = torch.empty((self.V, k_tab, w_ext), dtype=torch.int32, device=dev) if w_ext > 0 else None
+        self._check(self._lib.build_model_ngram_tables(self._h, _ptr(rows, torch.bfloat16), k_tab, w_ext, _ptr(tab),
+                                                       _ptr(val), _ptr(ext), _stream()), "build_model_ngram_tables")
+        self._keep_table = (tab, ext, rows)
+        return tab, val, ext
+
+    def set_model_table(self, tab: torch.Tensor, ext: torch.Tensor | None = None):
+        k_tab = int(tab.shape[1])
+        w_ext = int(ext.shape[2]) if ext is not None else 0
+        self._check(self._lib.spec_set_model_table(self._h, _ptr(tab, torch.int32), k_tab, _ptr(ext, torch.int32), w_ext),
+                    "spec_set_model_table")
+        self._keep_table = (tab, ext, None)
+
+    def draft_context_ngrams(self, hist: torch.Tensor, lens: torch.Tensor, qs, topk: int, B: int, w: int,
+                             flags: int = FLAG_DEDUP | FLAG_MODEL_FILL, out=None):
+        S, cap = int(hist.shape[0]), int(hist.shape[1])
+        dev = hist.device
+        if out is None:
+            out = (torch.empty((S, B, w), dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+                   torch.empty((S, B), dtype=torch.int32, device=dev), torch.empty((S, B), dtype=torch.int32, device=dev))
+        drafts, nd, src, counts = out
+        qs_arr = (C.c_int * max(1, len(qs)))(*[int(q) for q in qs])
+        self._check(self._lib.draft_context_ngrams(self._h, _ptr(hist, torch.int32), _ptr(lens, torch.int32), S, cap,
+                                                   qs_arr, len(qs), topk, B, w, flags, _ptr(drafts), _ptr(nd),
+                                                   _ptr(src), _ptr(counts), _stream()), "draft_context_ngrams")
+        return drafts, nd, src, counts
+
+    def verify_lmhead_argmax(self, hidden: torch.Tensor, out=None, with_max: bool = False):
+        M = int(hidden.shape[0])
+        if out is None:
+            out = (torch.empty(M, dtype=torch.int32, device=hidden.device),
+                   torch.empty(M, dtype=torch.float32, device=hidden.device) if with_max else None)
+        am, mx = out
+        self._check(self._lib.verify_lmhead_argmax(self._h, _ptr(hidden, torch.bfloat16), M, _ptr(am), _ptr(mx),
+                                                   _stream()), "verify_lmhead_argmax")
+        return am, mx
+
+    def accept_and_commit(self, drafts, n_drafts, argmax, hist, lens, out=None):
+        S, B, w = (int(x) for x in drafts.shape)
+        cap = int(hist.shape[1])
+        dev = hist.device
+        if out is None:
+            out = (torch.empty(S, dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+                   torch.empty((S, w + 1), dtype=torch.int32, device=dev))
+        acc, best, com = out
+        self._check(self._lib.accept_and_commit(self._h, _ptr(drafts, torch.int32), _ptr(n_drafts, torch.int32),
+                                                _ptr(argmax, torch.int32), S, B, w, _ptr(hist, torch.int32),
+                                                _ptr(lens, torch.int32), cap, _ptr(acc), _ptr(best), _ptr(com),
+                                                _stream()), "accept_and_commit")
+        return acc, best, com
+
+    def debug_logits(self, rows: torch.Tensor) -> torch.Tensor:
+        m = int(rows.shape[0])
+        out = torch.empty((m, self.V), dtype=torch.float32, device=rows.device)
+        self._check(self._lib.spec_debug_logits(self._h, _ptr(rows, torch.bfloat16), m, _ptr(out), _stream()),
+                    "spec_debug_logits")
+        return out

@@ -1,0 +1,668 @@
+// LM-head contraction Z = A * W^T on the 5th-generation tensor cores (tcgen05, accumulators in
+// TMEM, operands staged by TMA) with the row reduction fused into the epilogue, so Z never
+// reaches memory:
+//   MODE_ARGMAX  verification: per row of A the arg max over the vocabulary   (verify_lmhead_argmax)
+//   MODE_TOPK    model bigram table: per row the k largest entries           (build_model_ngram_tables)
+//   MODE_STORE   plain fp32 store, for the logits tolerance check            (spec_debug_logits)
+//
+// A is [a_rows, d] and W is [V, d], both bf16 and K-major, so both operands use the same
+// 128-byte-swizzled K-major shared-memory layout.  One CTA owns the accumulator of a
+// 128 x (<=256) tile: TMEM lane = row of A, TMEM column = vocabulary entry.  An epilogue thread
+// therefore owns one row of A and walks its columns in ascending vocabulary order, which makes
+// "lowest token id wins ties" a matter of using a strict comparison.
+//
+// Work is cut into units (m_tile, vocabulary chunk).  A persistent CTA takes units u, u + grid,
+// ...; inside a unit it sweeps the chunk in tiles of up to 256 columns and keeps the running
+// reduction in registers, then flushes once: a 64-bit atomicMax of (value, ~index) for the arg
+// max, a partial list for the top-k.  Small M (memory-bound: every SM streams its own slice of
+// W exactly once) and large M (tensor-bound) are the same kernel with different unit shapes.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (+ TMEM allocation), warp 1 = MMA issuer,
+// warps 2..5 = epilogue (TMEM lane quadrant = warp % 4).  Every wait on an mbarrier is bounded:
+// on expiry the CTA raises SPEC_STATUS_TIMEOUT, stops issuing work, and still frees its TMEM.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include <algorithm>
+#include <map>
+#include <tuple>
+#include <vector>
+
+#include "common.cuh"
+
+namespace ngs {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;               // 64 bf16 = one 128-byte swizzle row
+constexpr int BOX_N = 32;                 // rows of W per TMA box
+constexpr int MAX_BOXES = 8;              // up to 256 columns per tile
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;          // 16 KB
+constexpr int BOX_BYTES = BOX_N * BLOCK_K * 2;          // 4 KB
+constexpr int B_BYTES = MAX_BOXES * BOX_BYTES;          // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // 48 KB
+constexpr int ACC_COLS = 256;                           // TMEM columns per accumulator stage
+constexpr int TMEM_COLS = 512;
+constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+enum { MODE_ARGMAX = 0, MODE_TOPK = 1, MODE_STORE = 2 };
+
+struct GemmParams {
+    int a_rows;    // rows of A
+    int V;         // rows of W
+    int num_kb;    // ceil(d / 64)
+    int n_mtiles;  // ceil(a_rows / 128)
+    int n_boxes;   // ceil(V / 32)
+    int n_chunks;  // vocabulary chunks per m-tile
+    int align;     // chunk boundaries fall on multiples of `align` boxes
+    int group;     // m-tiles that run side by side (L2 reuse of the W chunk)
+    unsigned long long* keys;
+    unsigned int* ticket;
+    int32_t* argmax;
+    float* maxv;
+    int k_tab;
+    float* part_val;   // [n_chunks, a_rows, k_tab]
+    int32_t* part_idx;
+    float* logits;     // [a_rows, V]
+    int* status;
+};
+
+// ------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, one K = 16 slice.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B apart, 8-row
+// groups 1024 B apart (stride byte offset), descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr) {
+    uint64_t desc = 0;
+    desc |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+    desc |= (uint64_t)1 << 16;                     // leading byte offset (unused for swizzled K-major)
+    desc |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset
+    desc |= (uint64_t)1 << 46;                     // descriptor version
+    desc |= (uint64_t)2 << 61;                     // SWIZZLE_128B
+    return desc;
+}
+// Instruction descriptor for kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N given.
+__device__ __forceinline__ uint32_t make_idesc_bf16(int n_cols) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
+}
+
+// Order-preserving map of fp32 onto unsigned integers; key 0 lies below every real value.
+__device__ __forceinline__ uint32_t orderable_f32(float v) {
+    uint32_t u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_orderable_f32(uint32_t u) {
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
+}
+
+// ------------------------------------------------------------------------------------------ work units
+struct Unit {
+    int m_tile, chunk, box_begin, box_end;
+};
+__device__ __forceinline__ Unit decode_unit(const GemmParams& p, int u) {
+    Unit r;
+    const int per_group = p.group * p.n_chunks;
+    const int mg = u / per_group;
+    const int g = min(p.group, p.n_mtiles - mg * p.group);
+    const int local = u - mg * per_group;
+    r.chunk = local / g;
+    r.m_tile = mg * p.group + (local - r.chunk * g);
+    const long long n_al = (p.n_boxes + p.align - 1) / p.align;
+    r.box_begin = (int)((long long)r.chunk * n_al / p.n_chunks) * p.align;
+    r.box_end = min(p.n_boxes, (int)((long long)(r.chunk + 1) * n_al / p.n_chunks) * p.align);
+    return r;
+}
+
+// ------------------------------------------------------------------------------------------ the kernel
+template <int MODE>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;               // operand stages, 1024-byte aligned
+    unsigned char* tiles_ptr = smem_raw + (tiles - raw);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES);
+    // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * STAGES;
+    const uint32_t bar_tfull = bar_empty + 8 * STAGES;
+    const uint32_t bar_tempty = bar_tfull + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* is_last = reinterpret_cast<int*>(tmem_slot + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_units = p.n_mtiles * p.n_chunks;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull + 8 * a, 1);
+            mbar_init(bar_tempty + 8 * a, 4);
+        }
+        *abort_flag = 0;
+        *is_last = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+                const Unit un = decode_unit(p, u);
+                for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES) {
+                    const int nb = min(MAX_BOXES, un.box_end - b0);
+                    for (int kb = 0; kb < p.num_kb; ++kb) {
+                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t full = bar_full + 8 * stage;
+                        const uint32_t sa = tiles + stage * STAGE_BYTES;
+                        mbar_expect_tx(full, (uint32_t)(A_BYTES + nb * BOX_BYTES));
+                        tma_load_2d(sa, &tmA, kb * BLOCK_K, un.m_tile * BLOCK_M, full);
+                        for (int j = 0; j < nb; ++j)
+                            tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, kb * BLOCK_K, (b0 + j) * BOX_N, full);
+                        ++issued;
+                        if (++stage == STAGES) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                // Aborting: give copies already in flight a bounded chance to land before the CTA exits.
+                const int pending = issued < STAGES ? (int)issued : STAGES;
+                for (int i = 1; i <= pending; ++i) {
+                    int s2 = stage - i;
+                    uint32_t ph = phase;
+                    if (s2 < 0) {
+                        s2 += STAGES;
+                        ph ^= 1u;
+                    }
+                    for (int it = 0; it < 100000; ++it)
+                        if (mbar_try_wait(bar_full + 8 * s2, ph)) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t tile = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+                const Unit un = decode_unit(p, u);
+                for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
+                    const int nb = min(MAX_BOXES, un.box_end - b0);
+                    const uint32_t as = tile & 1u, aphase = (tile >> 1) & 1u;
+                    if (!mbar_wait(bar_tempty + 8 * as, aphase ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t idesc = make_idesc_bf16(nb * BOX_N);
+                    const uint32_t d_tmem = tmem_base + as * ACC_COLS;
+                    for (int kb = 0; kb < p.num_kb; ++kb) {
+                        if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t sa = tiles + stage * STAGE_BYTES;
+                        const uint64_t adesc = make_kmajor_sw128_desc(sa);
+                        const uint64_t bdesc = make_kmajor_sw128_desc(sa + A_BYTES);
+#pragma unroll
+                        for (int k = 0; k < BLOCK_K / 16; ++k)  // +32 bytes (2 x 16 B) per K = 16 slice
+                            tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        tc_commit(bar_empty + 8 * stage);  // frees the stage once these MMAs have read it
+                        if (++stage == STAGES) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                    if (ok) tc_commit(bar_tfull + 8 * as);  // accumulator complete
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (4 warps)
+        const int quad = warp & 3;
+        const int row_in_tile = quad * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
+        uint32_t tile = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+            const Unit un = decode_unit(p, u);
+            const int row = un.m_tile * BLOCK_M + row_in_tile;
+            // running reduction of this row over the unit's columns
+            float best_v = -INFINITY;
+            int best_i = 0x7FFFFFFF;
+            float tv[MODE == MODE_TOPK ? kMaxKTab : 1];
+            int ti[MODE == MODE_TOPK ? kMaxKTab : 1];
+            float thr = -INFINITY;
+            if (MODE == MODE_TOPK) {
+                for (int j = 0; j < p.k_tab; ++j) {
+                    tv[j] = -INFINITY;
+                    ti[j] = 0x7FFFFFFF;
+                }
+            }
+            for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
+                const int nb = min(MAX_BOXES, un.box_end - b0);
+                const uint32_t as = tile & 1u, aphase = (tile >> 1) & 1u;
+                if (!mbar_wait(bar_tfull + 8 * as, aphase, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const int col0 = b0 * BOX_N;
+                const int n_valid = min(nb * BOX_N, p.V - col0);
+                for (int c = 0; c < nb; ++c) {
+                    if (c * 32 >= n_valid) break;
+                    uint32_t r[32];
+                    __syncwarp();
+                    tmem_ld32(lane_base + as * ACC_COLS + c * 32, r);
+                    tmem_wait_ld();
+                    const int cbase = col0 + c * 32;
+                    const int lim = n_valid - c * 32;  // >= 1
+                    if (MODE == MODE_ARGMAX) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float v = __uint_as_float(r[j]);
+                            if (j < lim && v > best_v) {
+                                best_v = v;
+                                best_i = cbase + j;
+                            }
+                        }
+                    } else if (MODE == MODE_TOPK) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float v = __uint_as_float(r[j]);
+                            if (j < lim && v > thr) {
+                                int pos = p.k_tab - 1;
+                                while (pos > 0 && v > tv[pos - 1]) {
+                                    tv[pos] = tv[pos - 1];
+                                    ti[pos] = ti[pos - 1];
+                                    --pos;
+                                }
+                                tv[pos] = v;
+                                ti[pos] = cbase + j;
+                                thr = tv[p.k_tab - 1];
+                            }
+                        }
+                    } else {
+                        if (row < p.a_rows) {
+                            float* out = p.logits + (size_t)row * p.V + cbase;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < lim) out[j] = __uint_as_float(r[j]);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * as);
+            }
+            if (!ok) break;
+            if (row < p.a_rows) {
+                if (MODE == MODE_ARGMAX) {
+                    const unsigned long long key =
+                        ((unsigned long long)orderable_f32(best_v) << 32) | (unsigned long long)(~(uint32_t)best_i);
+                    atomicMax(p.keys + row, key);
+                } else if (MODE == MODE_TOPK) {
+                    const size_t base = ((size_t)un.chunk * p.a_rows + row) * p.k_tab;
+                    for (int j = 0; j < p.k_tab; ++j) {
+                        p.part_val[base + j] = tv[j];
+                        p.part_idx[base + j] = ti[j];
+                    }
+                }
+            }
+        }
+        if (MODE == MODE_ARGMAX) {
+            // The CTA that finishes last turns the merged keys into the outputs and re-arms the scratch.
+            const int et = threadIdx.x - 64;
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (et == 0) {
+                const unsigned int t = atomicAdd(p.ticket, 1u);
+                *is_last = (t == gridDim.x - 1) ? 1 : 0;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (*is_last) {
+                __threadfence();
+                for (int i = et; i < p.a_rows; i += 128) {
+                    const unsigned long long key = atomicExch(p.keys + i, 0ull);
+                    int idx = (int)(~(uint32_t)(key & 0xFFFFFFFFull));
+                    if (idx < 0 || idx >= p.V) idx = 0;
+                    p.argmax[i] = idx;
+                    if (p.maxv) p.maxv[i] = from_orderable_f32((uint32_t)(key >> 32));
+                }
+                if (et == 0) *p.ticket = 0u;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, SPEC_STATUS_TIMEOUT);
+    if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+// ------------------------------------------------------------------------------------------ table merge / extension
+// One thread per token x: merge the per-chunk partial lists (value descending, then token id
+// ascending) into the final k_tab entries.
+__global__ void merge_topk_kernel(const float* __restrict__ part_val, const int32_t* __restrict__ part_idx, int n_chunks,
+                                  int rows, int k, int32_t* __restrict__ tab_idx, float* __restrict__ tab_val) {
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= rows) return;
+    float tv[kMaxKTab];
+    int ti[kMaxKTab];
+    for (int j = 0; j < k; ++j) {
+        tv[j] = -INFINITY;
+        ti[j] = 0x7FFFFFFF;
+    }
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t base = ((size_t)c * rows + x) * k;
+        for (int j = 0; j < k; ++j) {
+            const float v = part_val[base + j];
+            const int i = part_idx[base + j];
+            if (i == 0x7FFFFFFF) break;
+            if (v > tv[k - 1] || (v == tv[k - 1] && i < ti[k - 1])) {
+                int pos = k - 1;
+                while (pos > 0 && (v > tv[pos - 1] || (v == tv[pos - 1] && i < ti[pos - 1]))) {
+                    tv[pos] = tv[pos - 1];
+                    ti[pos] = ti[pos - 1];
+                    --pos;
+                }
+                tv[pos] = v;
+                ti[pos] = i;
+            } else {
+                break;  // a chunk's list is sorted: nothing further in it can enter
+            }
+        }
+    }
+    for (int j = 0; j < k; ++j) {
+        tab_idx[(size_t)x * k + j] = ti[j] == 0x7FFFFFFF ? 0 : ti[j];
+        if (tab_val) tab_val[(size_t)x * k + j] = tv[j];
+    }
+}
+
+// ext[x][r][0] = T[x][r]; ext[x][r][j+1] = T[ext[x][r][j]][0].
+__global__ void extend_table_kernel(const int32_t* __restrict__ tab, int V, int k, int w, int32_t* __restrict__ ext) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)V * k) return;
+    int s = tab[i];
+    for (int j = 0; j < w; ++j) {
+        ext[i * w + j] = s;
+        s = (s >= 0 && s < V) ? tab[(size_t)s * k] : 0;
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host: unit shapes
+struct Shape {
+    int n_chunks, align, group, grid;
+};
+
+// Static-striding makespan of a candidate split, in boxes (a tile costs its boxes plus a fixed overhead).
+static double makespan(int n_mtiles, int n_boxes, int n_chunks, int align, int group, int grid) {
+    std::vector<double> load((size_t)grid, 0.0);
+    const long long n_al = (n_boxes + align - 1) / align;
+    const int per_group = group * n_chunks;
+    const int n_units = n_mtiles * n_chunks;
+    for (int u = 0; u < n_units; ++u) {
+        const int mg = u / per_group;
+        const int g = std::min(group, n_mtiles - mg * group);
+        const int chunk = (u - mg * per_group) / g;
+        const int b0 = (int)((long long)chunk * n_al / n_chunks) * align;
+        const int b1 = std::min(n_boxes, (int)((long long)(chunk + 1) * n_al / n_chunks) * align);
+        const int boxes = b1 - b0;
+        const int tiles = (boxes + MAX_BOXES - 1) / MAX_BOXES;
+        load[(size_t)(u % grid)] += boxes + 0.75 * tiles + 0.25;
+    }
+    double mx = 0;
+    for (double v : load) mx = std::max(mx, v);
+    return mx;
+}
+
+static Shape choose_shape(int n_mtiles, int n_boxes, int sms, int max_chunks) {
+    Shape best{1, 1, 1, 1};
+    double best_cost = 1e300;
+    const int group = std::min(n_mtiles, 8);
+    const int n_tiles = (n_boxes + MAX_BOXES - 1) / MAX_BOXES;
+    for (int align = 1; align <= MAX_BOXES; align += MAX_BOXES - 1) {
+        const int limit = std::min(max_chunks, align == 1 ? n_boxes : n_tiles);
+        for (int c = 1; c <= limit; ++c) {
+            // fine-grained (align 1) splits only make sense while a chunk is at most one tile
+            if (align == 1 && (n_boxes + c - 1) / c > MAX_BOXES && c > 1) continue;
+            const int units = n_mtiles * c;
+            const int grid = std::min(units, sms);
+            const double cost = makespan(n_mtiles, n_boxes, c, align, group, grid) * (1.0 + 1e-4 * c);
+            if (cost < best_cost) {
+                best_cost = cost;
+                best = Shape{c, align, group, grid};
+            }
+        }
+    }
+    return best;
+}
+
+static Shape cached_shape(spec_ctx* ctx, int n_mtiles, int n_boxes, int max_chunks) {
+    static std::map<std::tuple<int, int, int, int>, Shape> cache;
+    const auto key = std::make_tuple(n_mtiles, n_boxes, ctx->num_sms, max_chunks);
+    auto it = cache.find(key);
+    if (it != cache.end()) return it->second;
+    Shape s = choose_shape(n_mtiles, n_boxes, ctx->num_sms, max_chunks);
+    cache[key] = s;
+    return s;
+}
+
+template <int MODE>
+static int set_smem_attr(spec_ctx* ctx) {
+    static bool done[64] = {false};
+    bool& d = done[ctx->device & 63];
+    if (d) return SPEC_OK;
+    int rc = check_cuda(ctx, cudaFuncSetAttribute(head_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM),
+                        "head gemm: cudaFuncSetAttribute");
+    if (rc == SPEC_OK) d = true;
+    return rc;
+}
+
+static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& sh) {
+    p.a_rows = a_rows;
+    p.V = ctx->V;
+    p.num_kb = (ctx->d + BLOCK_K - 1) / BLOCK_K;
+    p.n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
+    p.n_boxes = (ctx->V + BOX_N - 1) / BOX_N;
+    p.n_chunks = sh.n_chunks;
+    p.align = sh.align;
+    p.group = sh.group;
+    p.keys = ctx->d_keys;
+    p.ticket = ctx->d_ticket;
+    p.argmax = nullptr;
+    p.maxv = nullptr;
+    p.k_tab = 0;
+    p.part_val = nullptr;
+    p.part_idx = nullptr;
+    p.logits = nullptr;
+    p.status = ctx->d_status;
+}
+
+int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st) {
+    int rc = set_smem_attr<MODE_ARGMAX>(ctx);
+    if (rc) return rc;
+    CUtensorMap tmA;
+    if ((rc = make_tensor_map(ctx, &tmA, d_hidden, M, ctx->d, BLOCK_M))) return rc;
+    const int n_mtiles = (M + BLOCK_M - 1) / BLOCK_M, n_boxes = (ctx->V + BOX_N - 1) / BOX_N;
+    const Shape sh = cached_shape(ctx, n_mtiles, n_boxes, 256);
+    GemmParams p;
+    fill_common(ctx, p, M, sh);
+    p.argmax = d_argmax;
+    p.maxv = d_max;
+    head_gemm_kernel<MODE_ARGMAX><<<sh.grid, GEMM_THREADS, GEMM_SMEM, st>>>(tmA, ctx->tm_unembed, p);
+    ctx->launches += 1;
+    return check_cuda(ctx, cudaGetLastError(), "verify_lmhead_argmax launch");
+}
+
+int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st) {
+    int rc = set_smem_attr<MODE_STORE>(ctx);
+    if (rc) return rc;
+    CUtensorMap tmA;
+    if ((rc = make_tensor_map(ctx, &tmA, d_rows, m, ctx->d, BLOCK_M))) return rc;
+    const int n_mtiles = (m + BLOCK_M - 1) / BLOCK_M, n_boxes = (ctx->V + BOX_N - 1) / BOX_N;
+    const Shape sh = cached_shape(ctx, n_mtiles, n_boxes, 256);
+    GemmParams p;
+    fill_common(ctx, p, m, sh);
+    p.logits = d_logits;
+    head_gemm_kernel<MODE_STORE><<<sh.grid, GEMM_THREADS, GEMM_SMEM, st>>>(tmA, ctx->tm_unembed, p);
+    ctx->launches += 1;
+    return check_cuda(ctx, cudaGetLastError(), "spec_debug_logits launch");
+}
+
+int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
+                 int32_t* d_ext, cudaStream_t st) {
+    int rc = set_smem_attr<MODE_TOPK>(ctx);
+    if (rc) return rc;
+    const int V = ctx->V;
+    CUtensorMap tmA;
+    if ((rc = make_tensor_map(ctx, &tmA, d_rows, V, ctx->d, BLOCK_M))) return rc;
+    const int n_mtiles = (V + BLOCK_M - 1) / BLOCK_M, n_boxes = (V + BOX_N - 1) / BOX_N;
+    // partial lists cost 8 bytes per entry and chunk: keep them under 256 MB
+    int max_chunks = (int)std::max<long long>(1, (256ll << 20) / ((long long)V * k_tab * 8));
+    max_chunks = std::min(max_chunks, 64);
+    const Shape sh = cached_shape(ctx, n_mtiles, n_boxes, max_chunks);
+    const size_t need = (size_t)sh.n_chunks * V * k_tab;
+    if (need > ctx->part_capacity) {
+        cudaStreamSynchronize(st);
+        cudaFree(ctx->d_part_val);
+        cudaFree(ctx->d_part_idx);
+        ctx->d_part_val = nullptr;
+        ctx->d_part_idx = nullptr;
+        ctx->part_capacity = 0;
+        if ((rc = check_cuda(ctx, cudaMalloc(&ctx->d_part_val, need * sizeof(float)), "cudaMalloc(partial values)"))) return rc;
+        if ((rc = check_cuda(ctx, cudaMalloc(&ctx->d_part_idx, need * sizeof(int32_t)), "cudaMalloc(partial ids)"))) return rc;
+        ctx->part_capacity = need;
+    }
+    GemmParams p;
+    fill_common(ctx, p, V, sh);
+    p.k_tab = k_tab;
+    p.part_val = ctx->d_part_val;
+    p.part_idx = ctx->d_part_idx;
+    head_gemm_kernel<MODE_TOPK><<<sh.grid, GEMM_THREADS, GEMM_SMEM, st>>>(tmA, ctx->tm_unembed, p);
+    if ((rc = check_cuda(ctx, cudaGetLastError(), "build_model_ngram_tables launch"))) return rc;
+    merge_topk_kernel<<<(V + 127) / 128, 128, 0, st>>>(ctx->d_part_val, ctx->d_part_idx, sh.n_chunks, V, k_tab, d_tab_idx,
+                                                      d_tab_val);
+    ctx->launches += 2;
+    if ((rc = check_cuda(ctx, cudaGetLastError(), "table merge launch"))) return rc;
+    if (d_ext) {
+        const long long n = (long long)V * k_tab;
+        extend_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d_tab_idx, V, k_tab, w_ext, d_ext);
+        ctx->launches += 1;
+        if ((rc = check_cuda(ctx, cudaGetLastError(), "table extension launch"))) return rc;
+    }
+    return SPEC_OK;
+}
+
+}  // namespace ngs

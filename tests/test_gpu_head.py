@@ -1,0 +1,128 @@
+"""GPU parity: tensor-core head (logits, verification argmax, model bigram table) vs the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from gpu_util import dev_bf16, dev_i32, weights
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2   # max-abs logit error allowed for bf16 inputs with fp32 accumulation
+
+
+@pytest.fixture(scope="module")
+def ngs():
+    import paper_2411_03786_b200 as m
+    return m
+
+
+def make_ctx(ngs, V, d, seed, std=1.0):
+    E = synth.gaussian_weights(V, d, std, seed, "E")
+    W = synth.gaussian_weights(V, d, std, seed, "W")
+    return E, W, ngs.SpecContext(dev_bf16(E), dev_bf16(W))
+
+
+# sizes span one tile, several tiles, ragged M / V / K tails
+SHAPES = [(1024, 128, 20), (1000, 200, 150), (4136, 320, 300), (96, 64, 1), (33, 8, 129)]
+
+
+@pytest.mark.parametrize("V,d,M", SHAPES)
+def test_logits_within_tolerance(ngs, V, d, M):
+    E, W, ctx = make_ctx(ngs, V, d, seed=V + d, std=d ** -0.5)
+    H = synth.hidden_literal(M, d, seed=M)
+    z = ctx.debug_logits(dev_bf16(H)).cpu().numpy().astype(np.float64)
+    ref = oracle.logits_rows(H, W)
+    assert z.shape == ref.shape
+    assert np.abs(z - ref).max() <= TOL
+    assert ctx.get_status() == 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("V,d,M", SHAPES)
+def test_verify_argmax_matches_oracle(ngs, V, d, M):
+    E, W, ctx = make_ctx(ngs, V, d, seed=V + d + 1, std=d ** -0.5)
+    H = synth.hidden_literal(M, d, seed=M + 1)
+    for rep in range(2):      # the second call checks that the merge scratch was re-armed
+        am, mx = ctx.verify_lmhead_argmax(dev_bf16(H), with_max=True)
+        am, mx = am.cpu().numpy(), mx.cpu().numpy().astype(np.float64)
+        ref_am, ref_mx, gap = oracle.verify(H, W)
+        bad = am != ref_am
+        assert not (bad & (gap >= TOL)).any(), f"{bad.sum()} mismatches with clear margins"
+        assert np.abs(mx - ref_mx).max() <= TOL
+    assert ctx.get_status() == 0
+    ctx.close()
+
+
+def test_verify_exact_ties_take_the_lowest_token(ngs):
+    V, d = 700, 64
+    W = synth.gaussian_weights(V, d, 1.0, 9, "W")
+    W[[40, 300, 650]] = W[5]               # identical rows in different tiles / chunks
+    ctx = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
+    H = W[[5, 650]].copy()
+    am, _ = ctx.verify_lmhead_argmax(dev_bf16(H))
+    assert am.cpu().tolist() == [5, 5]
+    ctx.close()
+
+
+def test_fp32_weights_are_rounded_once_like_the_oracle(ngs):
+    c = synth.config("C1")
+    E = synth.gaussian_weights(c["V"], c["d"], c["wstd"], 0, "E", "f32")
+    W = synth.gaussian_weights(c["V"], c["d"], c["wstd"], 0, "W", "f32")
+    ctx = ngs.SpecContext(torch.from_numpy(E).cuda(), torch.from_numpy(W).cuda())
+    Wb = oracle.round_to_bf16(W)
+    H = synth.hidden_literal(c["M"], c["d"], seed=0)
+    z = ctx.debug_logits(dev_bf16(H)).cpu().numpy().astype(np.float64)
+    assert np.abs(z - oracle.logits_rows(H, Wb)).max() <= TOL
+    # default table rows = the (rounded) embedding
+    tab, val, _ = ctx.build_model_ngram_tables(c["k_tab"], with_values=True)
+    check_table(tab.cpu().numpy(), val.cpu().numpy(), oracle.round_to_bf16(E), Wb, c["k_tab"], rows=None)
+    ctx.close()
+
+
+def check_table(tab, val, A, W, k, rows):
+    """epsilon-consistent top-k: ids distinct and in range; each rank's oracle logit within TOL of the
+    oracle's value at that rank; where the oracle's neighbouring gaps are clear the ids are identical."""
+    V = W.shape[0]
+    sel = np.arange(A.shape[0]) if rows is None else np.asarray(rows)
+    ref_idx, ref_val = oracle.model_table(A, W, k + 1 if k < V else k, rows=sel)
+    z = oracle.logits_rows(A, W, rows=sel)
+    n_same = 0
+    for n, x in enumerate(sel):
+        ids = tab[x]
+        assert len(set(ids.tolist())) == k and ids.min() >= 0 and ids.max() < V
+        assert np.abs(z[n, ids] - ref_val[n, :k]).max() <= TOL
+        assert np.abs(val[x] - z[n, ids]).max() <= TOL
+        gaps = ref_val[n, :-1] - ref_val[n, 1:]
+        if (gaps >= TOL).all():
+            assert np.array_equal(ids, ref_idx[n, :k])
+        n_same += int(np.array_equal(ids, ref_idx[n, :k]))
+    return n_same / len(sel)
+
+
+@pytest.mark.parametrize("V,d,k", [(1024, 128, 4), (1000, 200, 8), (4136, 64, 10), (300, 64, 32)])
+def test_model_table_matches_oracle(ngs, V, d, k):
+    E, W, ctx = make_ctx(ngs, V, d, seed=3 * V + d, std=1.0)
+    tab, val, ext = ctx.build_model_ngram_tables(k, w_ext=5, with_values=True)
+    tab, val, ext = tab.cpu().numpy(), val.cpu().numpy(), ext.cpu().numpy()
+    frac = check_table(tab, val, E, W, k, rows=None)
+    assert frac > 0.99
+    assert np.array_equal(ext, oracle.extend_table(tab, 5))       # integer stage: bit-exact given the same table
+    # caller-supplied rows (hidden state of every single-token context)
+    rows = synth.hidden_literal(V, d, seed=5)
+    tab2, val2, _ = ctx.build_model_ngram_tables(k, rows=dev_bf16(rows), with_values=True)
+    check_table(tab2.cpu().numpy(), val2.cpu().numpy(), rows, W, k, rows=None)
+    assert ctx.get_status() == 0
+    ctx.close()
+
+
+def test_table_ties_take_the_lower_token(ngs):
+    V, d = 300, 64
+    W = synth.gaussian_weights(V, d, 1.0, 4, "W")
+    W[[100, 200, 299]] = W[7]
+    ctx = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
+    tab, _, _ = ctx.build_model_ngram_tables(6)
+    ref, _ = oracle.model_table(W, W, 6, rows=[7, 299])
+    assert np.array_equal(tab.cpu().numpy()[[7, 299]], ref)
+    assert ref[0, :4].tolist() == [7, 100, 200, 299]
+    ctx.close()
