@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the batched N-gram speculation step on B200.
+
+One *step* = draft_context_ngrams -> verify_lmhead_argmax -> accept_and_commit over one batch of
+synthetic sequences (hidden states are an input: the transformer body is outside this library).
+The model bigram table is a one-off build and is timed separately (reported under "table_build").
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
+
+Prints ONE JSON line.  `--impl reference` times the plain CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+METRIC = "accepted_tokens_per_s"
+UNIT = "tokens/s"
+RHO = 0.55  # planted acceptance: P(accepted length >= j) = RHO^j  (about 2.2 tokens per call)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], tc_burst=d["bf16_tflops"], tc_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm=6650.0, tc_burst=1590.0, tc_sustained=1400.0, source="fallback")
+
+
+def host_inputs(c, rank):
+    """Seeded host-side inputs of one rank's batch (weights are shared, histories differ per rank)."""
+    seed = c["seed"]
+    E = synth.gaussian_weights(c["V"], c["d"], c["wstd"], seed, "E", c["wdtype"])
+    W = synth.gaussian_weights(c["V"], c["d"], c["wstd"], seed, "W", c["wdtype"])
+    cap = c["L"] + 64
+    hist, lens, copied = synth.zipf_histories(c["S"], c["L"], c["V"], c["zipf"], c["copy"], seed, cap=cap,
+                                              name=f"hist/rank{rank}")
+    return E, W, hist, lens, copied
+
+
+def bf16_bits(w):
+    return synth.f32_to_bf16_bits(w) if w.dtype == np.float32 else w
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self._stop = index, [], threading.Event()
+        self.t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout.strip()
+                if out:
+                    self.rows.append([x.strip() for x in out.splitlines()[0].split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self.t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self.t.join(timeout=6)
+
+    def summary(self):
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_step_time(c, hist, lens, T, H_bits, W_bits, budget_s, min_steps=1, max_steps=50):
+    """Times the oracle's step as it stands.  Verification is the costly part; when a full step would
+    exceed the budget the verify rows are sampled and the time is scaled to all M rows."""
+    import oracle
+    M = H_bits.shape[0]
+    t0 = time.perf_counter()
+    oracle.verify(H_bits, W_bits, rows=[0])
+    per_row = time.perf_counter() - t0
+    threads = oracle.num_threads()
+    est_full = per_row * M / max(1, min(threads, M))
+    rows = None
+    scale = 1.0
+    if est_full > budget_s / 2:
+        n = int(max(threads, min(M, (budget_s / 2) / per_row * threads)))
+        n = max(threads, n // threads * threads)
+        if n < M:
+            rows = np.linspace(0, M - 1, n).astype(np.int64)
+            scale = M / n
+    steps, total, accepted = 0, 0.0, 0
+    while steps < min_steps or (total < budget_s and steps < max_steps):
+        h, l = hist.copy(), lens.copy()
+        t0 = time.perf_counter()
+        drafts, nd, _, _ = oracle.draft_batch(h, l, c["qs"], c["topk"], c["B"], c["w"], 3, T)
+        t1 = time.perf_counter()
+        am, _, _ = oracle.verify(H_bits, W_bits, rows=rows)
+        t2 = time.perf_counter()
+        if rows is not None:
+            full = np.zeros(M, np.int32)
+            full[rows] = am
+            am = full
+        acc, _, _ = oracle.accept_commit(drafts, nd, am.reshape(c["S"], c["B"], c["w"] + 1), h, l)
+        t3 = time.perf_counter()
+        total += (t1 - t0) + (t2 - t1) * scale + (t3 - t2)
+        accepted += int((acc + 1).sum())
+        steps += 1
+    sample = (f"{steps} full oracle steps (draft + verify of all {M} rows + accept)" if rows is None else
+              f"{steps} oracle steps with verify on {len(rows)} of {M} rows, verify time scaled by {scale:.1f}")
+    return total / steps, accepted / steps, threads, sample, rows is not None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="C2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU work for the oracle baseline")
+    ap.add_argument("--no-table", action="store_true", help="skip timing the one-off table build")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    c = synth.config(args.workload)
+    cfg = {"workload": f"{args.workload}: V={c['V']} d={c['d']} S={c['S']} L={c['L']} qs={list(c['qs'])} topk={c['topk']} "
+                       f"B={c['B']} w={c['w']} M={c['M']} k_tab={c['k_tab']} per GPU",
+           "hidden_states": f"planted acceptance rho={RHO}", "l2": "verify streams the unembedding (larger than L2) every step; "
+           "draft/accept inputs are KB-sized and stay L2-resident", "sharding": "sequences per rank, no collective"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        return run_reference(args, c, cfg)
+
+    import torch
+    import paper_2411_03786_b200 as ngs
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    pk = peaks()
+
+    E, W, hist_h, lens_h, copied = host_inputs(c, rank)
+    to_dev = (lambda w: torch.from_numpy(w).to(dev)) if c["wdtype"] == "f32" else \
+        (lambda w: torch.from_numpy(w.view(np.int16)).view(torch.bfloat16).to(dev))
+    dE, dW = to_dev(E), to_dev(W)
+    ctx = ngs.SpecContext(dE, dW)
+    W_bits = bf16_bits(W)
+
+    # ---- one-off table build (timed on its own)
+    table = {}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    tab, _, ext = ctx.build_model_ngram_tables(c["k_tab"], w_ext=c["w"])
+    torch.cuda.synchronize()
+    if not args.no_table:
+        reps = 3 if c["V"] <= 40000 else 1
+        ts = []
+        for _ in range(reps):
+            a, b = ev(), ev()
+            a.record()
+            ctx.build_model_ngram_tables(c["k_tab"], w_ext=c["w"])
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ms = min(ts)
+        fl = 2.0 * c["V"] * c["V"] * c["d"]
+        table = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_burst_peak": fl / ms / 1e9 / pk["tc_burst"],
+                 "frac_of_sustained_peak": fl / ms / 1e9 / pk["tc_sustained"], "flops": fl, "peak_source": pk["source"]}
+
+    # ---- inputs of a step: histories, then hidden states planted on the initial drafts
+    hist, lens0 = torch.from_numpy(hist_h).to(dev), torch.from_numpy(lens_h).to(dev)
+    lens = lens0.clone()
+    S, B, w, M = c["S"], c["B"], c["w"], c["M"]
+    out_d = ctx.draft_context_ngrams(hist, lens, c["qs"], c["topk"], B, w)
+    torch.cuda.synchronize()
+    drafts0, nd0 = out_d[0].cpu().numpy(), out_d[1].cpu().numpy()
+    targets, _, planted_a = synth.planted_targets(drafts0, nd0, None, c["V"], c["zipf"], RHO, seed=c["seed"] + 100 * rank)
+    H_bits = synth.hidden_planted(W_bits, targets.reshape(-1), seed=c["seed"] + 100 * rank)
+    dH = torch.from_numpy(H_bits.view(np.int16)).view(torch.bfloat16).to(dev)
+    out_v = (torch.empty(M, dtype=torch.int32, device=dev), None)
+    out_a = (torch.empty(S, dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+             torch.empty((S, w + 1), dtype=torch.int32, device=dev))
+
+    def step(timers=None):
+        lens.copy_(lens0)                      # every iteration sees the same history length
+        if timers:
+            timers[0].record()
+        ctx.draft_context_ngrams(hist, lens, c["qs"], c["topk"], B, w, out=out_d)
+        if timers:
+            timers[1].record()
+        ctx.verify_lmhead_argmax(dH, out=out_v)
+        if timers:
+            timers[2].record()
+        ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), hist, lens, out=out_a)
+        if timers:
+            timers[3].record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    launches0 = ctx.launch_count()
+    timers = [[ev() for _ in range(4)] for _ in range(args.steps)]
+    t_begin, t_end = ev(), ev()
+    with ClockSampler(local_rank) as clk:
+        barrier()
+        t_begin.record()
+        for i in range(args.steps):
+            step(timers[i])
+        t_end.record()
+        barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    launches = ctx.launch_count() - launches0
+    acc_mean = float((out_a[0].float() + 1).sum().item())          # tokens committed by one step of this rank
+    status = ctx.get_status()
+    phase = lambda a, b: statistics.mean(t[a].elapsed_time(t[b]) for t in timers)
+    draft_ms, verify_ms, accept_ms = phase(0, 1), phase(1, 2), phase(2, 3)
+
+    # ---- end to end through the public API with host buffers
+    pin = lambda t: t.cpu().pin_memory()
+    h_hist, h_lens, h_H = pin(hist), pin(lens0), pin(dH.view(torch.int16))
+    h_acc, h_com = torch.empty(S, dtype=torch.int32).pin_memory(), torch.empty((S, w + 1), dtype=torch.int32).pin_memory()
+    d_hist2, d_H2 = torch.empty_like(hist), torch.empty_like(dH.view(torch.int16))
+
+    def e2e_step():
+        d_hist2.copy_(h_hist, non_blocking=True)
+        lens.copy_(h_lens, non_blocking=True)
+        d_H2.copy_(h_H, non_blocking=True)
+        ctx.draft_context_ngrams(d_hist2, lens, c["qs"], c["topk"], B, w, out=out_d)
+        ctx.verify_lmhead_argmax(d_H2.view(torch.bfloat16), out=out_v)
+        ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), d_hist2, lens, out=out_a)
+        h_acc.copy_(out_a[0], non_blocking=True)
+        h_com.copy_(out_a[2], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e_begin, e_end = ev(), ev()
+    e_begin.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e_end.record()
+    barrier()
+    e2e_ms = e_begin.elapsed_time(e_end)
+    h2d = h_hist.numel() * 4 + h_lens.numel() * 4 + h_H.numel() * 2
+    d2h = h_acc.numel() * 4 + h_com.numel() * 4
+
+    # ---- max over ranks, totals over ranks
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms, verify_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms, verify_ms = (float(x) for x in t)
+        a = torch.tensor([acc_mean], device=dev, dtype=torch.float64)
+        dist.all_reduce(a, op=dist.ReduceOp.SUM)
+        acc_total = float(a[0])
+    else:
+        acc_total = acc_mean
+    ms_per_step = total_ms / args.steps
+    value = acc_total / (ms_per_step / 1e3)
+    e2e_value = acc_total / (e2e_ms / args.steps / 1e3)
+
+    # ---- roofline of the dominant kernel (the verify contraction)
+    bytes_alg = 2.0 * c["V"] * c["d"] + 2.0 * M * c["d"] + 4.0 * M
+    flops = 2.0 * M * c["V"] * c["d"]
+    t_hbm, t_tc = bytes_alg / (pk["hbm"] * 1e9), flops / (pk["tc_sustained"] * 1e12)
+    if t_hbm >= t_tc:
+        ach = bytes_alg / (verify_ms / 1e3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s", "frac": ach / pk["hbm"]}
+    else:
+        ach = flops / (verify_ms / 1e3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": pk["tc_sustained"], "unit": "TFLOP/s",
+                "frac": ach / pk["tc_sustained"]}
+    roof.update({"traffic": TRAFFIC.get(args.workload), "kernel": "head_gemm_kernel<ARGMAX> (verify_lmhead_argmax)",
+                 "ms_per_launch": verify_ms, "algorithmic_bytes": bytes_alg, "flops": flops,
+                 "peak_source": pk["source"] + (" sustained" if roof["bound"] == "tensor" else " copy")})
+
+    line = None
+    if rank == 0:
+        cpu = {}
+        if world == 1 or rank == 0:
+            T_h = tab.cpu().numpy()
+            sec, acc_cpu, threads, sample, sampled = oracle_step_time(c, hist_h, lens_h, T_h, H_bits, W_bits, args.cpu_budget)
+            cpu = {"value": acc_cpu / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                   "s_per_step": sec}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic", "config": cfg,
+                "steps_per_s": world * 1e3 / ms_per_step, "tokens_per_step": acc_total / world / S,
+                "phase_ms": {"draft": draft_ms, "verify": verify_ms, "accept": accept_ms},
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "ms_per_step": e2e_ms / args.steps},
+                "gpu_launches": int(launches), "roofline": roof, "table_build": table, "cpu_baseline": cpu,
+                "clocks": clk.summary(), "status_bits": status, "copied_fraction": copied}
+        print(json.dumps(line))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+# DRAM bytes per verify launch from the ncu captures summarised under profiles/ (None = not captured
+# for the current kernel).
+TRAFFIC = {}
+
+
+def run_reference(args, c, cfg):
+    """The CPU oracle, as it stands, on the host cores: same workload, metric and unit."""
+    import oracle
+    E, W, hist_h, lens_h, _ = host_inputs(c, 0)
+    W_bits = bf16_bits(W)
+    k = c["k_tab"]
+    # a model table is an input of the step; rank-order rows of it are irrelevant to the timing, so a
+    # seeded stand-in is used instead of the (hours-long) CPU table build
+    g = synth.stream(c["seed"], "ref/T")
+    T = g.integers(0, c["V"], (c["V"], k)).astype(np.int32)
+    drafts0, nd0, _, _ = oracle.draft_batch(hist_h, lens_h, c["qs"], c["topk"], c["B"], c["w"], 3, T)
+    targets, _, _ = synth.planted_targets(drafts0, nd0, None, c["V"], c["zipf"], RHO, seed=c["seed"])
+    H_bits = synth.hidden_planted(W_bits, targets.reshape(-1), seed=c["seed"])
+    per_step_budget = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(min(args.warmup, 1)):
+        oracle_step_time(c, hist_h, lens_h, T, H_bits, W_bits, per_step_budget, max_steps=1)
+    secs, accs = [], []
+    t_wall = time.perf_counter()
+    for _ in range(args.steps):
+        sec, acc, threads, sample, _ = oracle_step_time(c, hist_h, lens_h, T, H_bits, W_bits, per_step_budget, max_steps=1)
+        secs.append(sec)
+        accs.append(acc)
+        if time.perf_counter() - t_wall > 150:
+            break
+    sec = statistics.mean(secs)
+    value = statistics.mean(accs) / sec
+    cpu = {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+                      "steps": len(secs), "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+                      "cpu_baseline": cpu, "gpu_launches": 0,
+                      "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
