@@ -58,6 +58,7 @@ enum {
 enum { SPEC_F32 = 0, SPEC_BF16 = 1 };
 enum { SPEC_FLAG_DEDUP = 1, SPEC_FLAG_MODEL_FILL = 2 };
 enum { SPEC_MAX_VERIFY_ROWS = 65536 };
+enum { SPEC_NOALLOC_MAX_ROWS = 4096 }; /* row limit of verify_lmhead_argmax_noalloc */
 
 /*
  * Create a context for one model head on one device.
@@ -148,6 +149,34 @@ int accept_and_commit(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_n
  * d_logits[i, y] = <rows[i, :], unembed[y, :]> for i < m, as float32 [m, V].
  */
 int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, void* stream);
+
+/*
+ * Verification head for callers that must not allocate.  (The paper has no counterpart: this is
+ * a packaging variant of verify_lmhead_argmax, same kernel, same result.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they verify drafts: a
+ * serving engine that has already handed all device memory to its own pool, a plug-in invoked
+ * where an allocation's implicit device-wide synchronisation would stall other streams, or code
+ * that is simply forbidden to change the memory map at run time.  Such callers cannot create a
+ * context (spec_init allocates), so this entry point takes the unembedding matrix directly and
+ * keeps its cross-CTA merge scratch in a fixed array inside the library image instead.
+ *
+ *   d_unembed  [V, d] bfloat16 lm_head weight, borrowed.   d_hidden [M, d] bfloat16.
+ *   d_argmax   [M] int32 out.   d_max [M] float32 out or NULL.   device = CUDA ordinal.
+ *
+ *   - M may not exceed SPEC_NOALLOC_MAX_ROWS; a larger M is rejected with SPEC_ERR_ARG.  The array
+ *     (about 33 KB) is held by every GPU that loads the library, until the process exits.
+ *   - It calls no cudaMalloc / cudaFree and no allocating routine; it enqueues three small memsets
+ *     and one kernel on `stream`.
+ *   - The first call on each device looks up the array's device address and the driver's
+ *     tensor-map encoder; make that first call before any stream capture begins.
+ *   - All calls share the one array and it keeps the previous call's contents, so the call clears
+ *     what it needs first.  Two calls whose GPU work overlaps (different streams, or different
+ *     threads) race on it: serialise them.
+ *   - d_argmax is pre-set to -1; if a bounded device-side wait ever expired the rows stay -1.
+ */
+int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d, const void* d_hidden, int M,
+                                 int32_t* d_argmax, float* d_max, int device, void* stream);
 
 /* Number of kernels the library has launched for this context since spec_init. */
 long long spec_launch_count(spec_ctx* ctx);

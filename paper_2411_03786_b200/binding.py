@@ -51,6 +51,7 @@ def load_library(build: bool = True) -> C.CDLL:
     lib.accept_and_commit.argtypes = [vp, i32p, i32p, i32p, C.c_int, C.c_int, C.c_int, i32p, i32p, C.c_int, i32p,
                                       i32p, i32p, vp]
     lib.spec_debug_logits.argtypes = [vp, vp, C.c_int, fp, vp]
+    lib.verify_lmhead_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, i32p, fp, C.c_int, vp]
     lib.spec_launch_count.argtypes = [vp]
     lib.spec_launch_count.restype = C.c_longlong
     _lib = lib
@@ -173,3 +174,21 @@ class SpecContext:
         self._check(self._lib.spec_debug_logits(self._h, _ptr(rows, torch.bfloat16), m, _ptr(out), _stream()),
                     "spec_debug_logits")
         return out
+
+
+def verify_lmhead_argmax_noalloc(unembed: torch.Tensor, hidden: torch.Tensor, out):
+    """Context-free verification for callers that must not allocate device memory.
+
+    ``out = (argmax int32 [M], max float32 [M] or None)`` must be preallocated by the caller: this
+    wrapper allocates nothing either.  See ``verify_lmhead_argmax_noalloc`` in the header for the
+    row limit and the rule that calls must not overlap on the GPU.
+    """
+    lib = load_library()
+    am, mx = out
+    V, d = int(unembed.shape[0]), int(unembed.shape[1])
+    rc = lib.verify_lmhead_argmax_noalloc(_ptr(unembed, torch.bfloat16), V, d, _ptr(hidden, torch.bfloat16),
+                                          int(hidden.shape[0]), _ptr(am, torch.int32), _ptr(mx), unembed.device.index or 0,
+                                          _stream())
+    if rc != 0:
+        raise SpecError(f"verify_lmhead_argmax_noalloc failed ({rc}): {lib.spec_last_error(None).decode()}")
+    return am, mx

@@ -666,3 +666,83 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
 }
 
 }  // namespace ngs
+
+// ------------------------------------------------------------------------------------------ allocation-free verify
+// Scratch of verify_lmhead_argmax_noalloc: merge keys for SPEC_NOALLOC_MAX_ROWS rows, then one word
+// for the completion ticket and one for the status bits.  It lives in the library image, so every
+// GPU that loads the library holds these ~33 KB until the process exits.
+static __device__ __align__(256) unsigned long long g_noalloc_scratch[SPEC_NOALLOC_MAX_ROWS + 32];
+
+namespace ngs {
+struct NoAllocDevice {
+    bool ready = false;
+    unsigned long long* scratch = nullptr;  // device address of g_noalloc_scratch on this device
+    int num_sms = 0;
+    EncodeTiledFn encode = nullptr;
+};
+static NoAllocDevice g_noalloc_dev[64];
+}  // namespace ngs
+
+extern "C" int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d, const void* d_hidden, int M,
+                                            int32_t* d_argmax, float* d_max, int device, void* stream) {
+    using namespace ngs;
+    if (!d_unembed || !d_hidden || !d_argmax) return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax_noalloc: NULL pointer");
+    if (!aligned16(d_unembed) || !aligned16(d_hidden))
+        return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax_noalloc: matrices must be 16-byte aligned");
+    if (V <= 0 || d <= 0 || d % 8 != 0) return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax_noalloc: need V > 0, d > 0, d %% 8 == 0");
+    if (M < 0 || M > SPEC_NOALLOC_MAX_ROWS)
+        return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax_noalloc: M = %d exceeds the built-in scratch (at most %d rows); "
+                    "use verify_lmhead_argmax with a context for larger blocks", M, (int)SPEC_NOALLOC_MAX_ROWS);
+    if (device < 0 || device >= 64) return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax_noalloc: device %d out of range", device);
+    if (M == 0) return SPEC_OK;
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) return check_cuda(nullptr, e, "verify_lmhead_argmax_noalloc: cudaSetDevice");
+
+    NoAllocDevice& nd = g_noalloc_dev[device];
+    if (!nd.ready) {
+        // One-time set-up for this device (made current above).  In host code the array's name is only a
+        // handle: the address a kernel can use has to be asked for, per device.
+        int major = 0;
+        if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device)) != cudaSuccess)
+            return check_cuda(nullptr, e, "verify_lmhead_argmax_noalloc: cudaDeviceGetAttribute");
+        if (major != 10) return fail(nullptr, SPEC_ERR_CUDA, "verify_lmhead_argmax_noalloc: device %d is not sm_100", device);
+        if ((e = cudaDeviceGetAttribute(&nd.num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess)
+            return check_cuda(nullptr, e, "verify_lmhead_argmax_noalloc: cudaDeviceGetAttribute");
+        unsigned long long* ptr = nullptr;
+        if ((e = cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch)) != cudaSuccess || !ptr)
+            return check_cuda(nullptr, e == cudaSuccess ? cudaErrorInvalidSymbol : e, "verify_lmhead_argmax_noalloc: cudaGetSymbolAddress");
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess)
+            return fail(nullptr, SPEC_ERR_CUDA, "verify_lmhead_argmax_noalloc: cuTensorMapEncodeTiled not available from the driver");
+        nd.scratch = ptr;
+        nd.encode = (EncodeTiledFn)fn;
+        nd.ready = true;
+    }
+
+    // A context on the stack, pointing at the built-in scratch, lets the ordinary launch path run unchanged.
+    spec_ctx tmp;
+    tmp.device = device;
+    tmp.V = V;
+    tmp.d = d;
+    tmp.num_sms = nd.num_sms;
+    tmp.unembed = d_unembed;
+    tmp.encode = nd.encode;
+    tmp.d_keys = nd.scratch;
+    tmp.d_ticket = reinterpret_cast<unsigned int*>(nd.scratch + SPEC_NOALLOC_MAX_ROWS);
+    tmp.d_status = reinterpret_cast<int*>(nd.scratch + SPEC_NOALLOC_MAX_ROWS + 1);
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = make_tensor_map(&tmp, &tmp.tm_unembed, d_unembed, V, d, BOX_N);
+    if (rc == SPEC_OK) {
+        // The scratch keeps whatever the previous call left: the keys of this call's rows, the ticket and
+        // the status word must start at zero.  Outputs start at -1 so an expired wait cannot pass for a result.
+        e = cudaMemsetAsync(nd.scratch, 0, sizeof(unsigned long long) * (size_t)M, st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(nd.scratch + SPEC_NOALLOC_MAX_ROWS, 0, 2 * sizeof(unsigned long long), st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(d_argmax, 0xFF, sizeof(int32_t) * (size_t)M, st);
+        rc = check_cuda(&tmp, e, "verify_lmhead_argmax_noalloc: cudaMemsetAsync");
+    }
+    if (rc == SPEC_OK) rc = launch_verify(&tmp, d_hidden, M, d_argmax, d_max, st);
+    if (rc != SPEC_OK) return fail(nullptr, rc, "%s", tmp.err);
+    return SPEC_OK;
+}
