@@ -44,8 +44,8 @@ def peaks():
 def host_inputs(c, rank):
     """Seeded host-side inputs of one rank's batch (weights are shared, histories differ per rank)."""
     seed = c["seed"]
-    E = synth.gaussian_weights(c["V"], c["d"], c["wstd"], seed, "E", c["wdtype"])
-    W = synth.gaussian_weights(c["V"], c["d"], c["wstd"], seed, "W", c["wdtype"])
+    E = synth.gaussian_weights(c["V"], c["d"], c["wstd"], c["wseed"], "E", c["wdtype"])
+    W = synth.gaussian_weights(c["V"], c["d"], c["wstd"], c["wseed"], "W", c["wdtype"])
     cap = c["L"] + 64
     hist, lens, copied = synth.zipf_histories(c["S"], c["L"], c["V"], c["zipf"], c["copy"], seed, cap=cap,
                                               name=f"hist/rank{rank}")
@@ -316,7 +316,7 @@ def main():
     line = None
     if rank == 0:
         cpu = {}
-        if world == 1 or rank == 0:
+        if args.cpu_budget > 0:
             T_h = tab.cpu().numpy()
             sec, acc_cpu, threads, sample, sampled = oracle_step_time(c, hist_h, lens_h, T_h, H_bits, W_bits, args.cpu_budget)
             cpu = {"value": acc_cpu / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,

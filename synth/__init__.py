@@ -201,5 +201,7 @@ CONFIGS = {
 def config(name: str) -> dict:
     c = dict(CONFIGS[name])
     c["name"] = name
+    # C3 reuses C2's head (and table), C5 reuses C4's: weights are keyed by wseed
+    c["wseed"] = {"C3": CONFIGS["C2"]["seed"], "C5": CONFIGS["C4"]["seed"]}.get(name, c["seed"])
     c["M"] = c["S"] * c["B"] * (c["w"] + 1)
     return c

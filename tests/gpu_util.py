@@ -15,5 +15,5 @@ def dev_i32(a: np.ndarray) -> torch.Tensor:
 
 def weights(c, which):
     """bf16 bit patterns of a config's weight matrix (fp32 configs are rounded once, as the library does)."""
-    w = synth.gaussian_weights(c["V"], c["d"], c["wstd"], c["seed"], which, c["wdtype"])
+    w = synth.gaussian_weights(c["V"], c["d"], c["wstd"], c["wseed"], which, c["wdtype"])
     return synth.f32_to_bf16_bits(w) if c["wdtype"] == "f32" else w
