@@ -114,10 +114,11 @@ int spec_init(spec_ctx** out, const void* d_embed, const void* d_unembed, int dt
         cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st);
         cudaMemsetAsync(ctx->d_keys, 0, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS, st);
         cudaMemsetAsync(ctx->d_ticket, 0, sizeof(unsigned int), st);
-        if ((rc = make_tensor_map(ctx, &ctx->tm_unembed, ctx->unembed, V, d, 32))) {
+        if ((rc = make_tensor_map(ctx, &ctx->tm_w[1], ctx->unembed, V, d, 32))) {
             strncpy(g_err, ctx->err, 255);
             break;
         }
+        ctx->tm_w_ready[1] = true;
         if ((rc = check_cuda(nullptr, cudaStreamSynchronize(st), "spec_init: stream sync"))) break;
     } while (0);
     if (rc != SPEC_OK) {

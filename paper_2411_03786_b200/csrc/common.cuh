@@ -43,7 +43,10 @@ struct spec_ctx {
     const int32_t* ext = nullptr;
     int w_ext = 0;
     ngs::EncodeTiledFn encode = nullptr;
-    CUtensorMap tm_unembed;  // B operand of every contraction
+    // B operand of every contraction: tensor maps of the unembedding with 16/32/64/128/256-row boxes,
+    // encoded on first use (host-side work only)
+    CUtensorMap tm_w[5];
+    bool tm_w_ready[5] = {false, false, false, false, false};
     long long launches = 0;
     char err[256] = {0};
 };

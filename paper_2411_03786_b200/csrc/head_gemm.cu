@@ -11,8 +11,10 @@
 // therefore owns one row of A and walks its columns in ascending vocabulary order, which makes
 // "lowest token id wins ties" a matter of using a strict comparison.
 //
-// Work is cut into units (m_tile, vocabulary chunk).  A persistent CTA takes units u, u + grid,
-// ...; inside a unit it sweeps the chunk in tiles of up to 256 columns and keeps the running
+// Work is cut into units (m_tile, vocabulary chunk).  CTA b of the grid = group x slots works on
+// m-tile b % group of each m-group and on chunks b / group, + slots, ...: CTAs of one slot walk
+// the same chunks of W together, so W comes from HBM once per m-group.  Inside a unit the CTA
+// sweeps the chunk in tiles of up to 256 columns and keeps the running
 // reduction in registers, then flushes once: a 64-bit atomicMax of (value, ~index) for the arg
 // max, a partial list for the top-k.  Small M (memory-bound: every SM streams its own slice of
 // W exactly once) and large M (tensor-bound) are the same kernel with different unit shapes.
@@ -22,6 +24,7 @@
 // on expiry the CTA raises SPEC_STATUS_TIMEOUT, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
 #include <math.h>
+#include <stdlib.h>
 
 #include <algorithm>
 #include <map>
@@ -34,17 +37,14 @@ namespace ngs {
 
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;               // 64 bf16 = one 128-byte swizzle row
-constexpr int BOX_N = 32;                 // rows of W per TMA box
-constexpr int MAX_BOXES = 8;              // up to 256 columns per tile
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;          // 16 KB
-constexpr int BOX_BYTES = BOX_N * BLOCK_K * 2;          // 4 KB
-constexpr int B_BYTES = MAX_BOXES * BOX_BYTES;          // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // 48 KB
+constexpr int TILE_N = 256;               // up to 256 columns (rows of W) per tile, in boxes of 16..256 rows
+constexpr int MAX_STAGES = 8;
+constexpr int A_TILE_BYTES = BLOCK_M * BLOCK_K * 2;     // 16 KB: what one MMA reads of A
+constexpr int SMEM_LIMIT = 227 * 1024;                  // dynamic shared memory per CTA on sm_100
+constexpr int SMEM_MISC = 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int ACC_COLS = 256;                           // TMEM columns per accumulator stage
 constexpr int TMEM_COLS = 512;
 constexpr int GEMM_THREADS = 192;
-constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum { MODE_ARGMAX = 0, MODE_TOPK = 1, MODE_STORE = 2 };
@@ -54,10 +54,16 @@ struct GemmParams {
     int V;         // rows of W
     int num_kb;    // ceil(d / 64)
     int n_mtiles;  // ceil(a_rows / 128)
-    int n_boxes;   // ceil(V / 32)
+    int box_n;     // rows of W per TMA box (16, 32, 64, 128 or 256)
+    int n_boxes;   // ceil(V / box_n)
     int n_chunks;  // vocabulary chunks per m-tile
-    int align;     // chunk boundaries fall on multiples of `align` boxes
-    int group;     // m-tiles that run side by side (L2 reuse of the W chunk)
+    int group;     // m-tiles that run side by side on the same W chunk (L2 reuse)
+    int n_groups;  // ceil(n_mtiles / group)
+    int n_slots;   // grid = group * n_slots
+    int a_box_rows;   // rows of A per TMA box (128, or fewer when A has fewer rows)
+    int a_bytes;      // shared-memory bytes reserved for the A tile of a stage (multiple of 1024)
+    int stage_bytes;  // a_bytes + boxes per tile * box bytes
+    int stages;       // depth of the operand ring
     unsigned long long* keys;
     unsigned int* ticket;
     int32_t* argmax;
@@ -185,40 +191,53 @@ __device__ __forceinline__ float from_orderable_f32(uint32_t u) {
 struct Unit {
     int m_tile, chunk, box_begin, box_end;
 };
-__device__ __forceinline__ Unit decode_unit(const GemmParams& p, int u) {
-    Unit r;
-    const int per_group = p.group * p.n_chunks;
-    const int mg = u / per_group;
-    const int g = min(p.group, p.n_mtiles - mg * p.group);
-    const int local = u - mg * per_group;
-    r.chunk = local / g;
-    r.m_tile = mg * p.group + (local - r.chunk * g);
-    const long long n_al = (p.n_boxes + p.align - 1) / p.align;
-    r.box_begin = (int)((long long)r.chunk * n_al / p.n_chunks) * p.align;
-    r.box_end = min(p.n_boxes, (int)((long long)(r.chunk + 1) * n_al / p.n_chunks) * p.align);
-    return r;
-}
+// Units of this CTA in execution order.
+struct UnitIter {
+    int mg, c, mi, slot;
+    __device__ __forceinline__ explicit UnitIter(const GemmParams& p)
+        : mg(0), c((int)blockIdx.x / p.group), mi((int)blockIdx.x % p.group), slot((int)blockIdx.x / p.group) {}
+    __device__ __forceinline__ bool next(const GemmParams& p, Unit& u) {
+        while (mg < p.n_groups) {
+            const int m_tile = mg * p.group + mi;
+            if (m_tile < p.n_mtiles && c < p.n_chunks) {
+                u.m_tile = m_tile;
+                u.chunk = c;
+                u.box_begin = (int)((long long)c * p.n_boxes / p.n_chunks);
+                u.box_end = (int)((long long)(c + 1) * p.n_boxes / p.n_chunks);
+                c += p.n_slots;
+                return true;
+            }
+            ++mg;
+            c = slot;
+        }
+        return false;
+    }
+};
 
 // ------------------------------------------------------------------------------------------ the kernel
-template <int MODE>
+// KT = capacity of the per-thread top-k list (registers); only MODE_TOPK uses it.
+template <int MODE, int KT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;               // operand stages, 1024-byte aligned
     unsigned char* tiles_ptr = smem_raw + (tiles - raw);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES);
+    const int STAGES = p.stages, STAGE_BYTES = p.stage_bytes, A_BYTES = p.a_bytes;
+    const int BOX_N = p.box_n, BOX_BYTES = p.box_n * BLOCK_K * 2, MAX_BOXES = TILE_N / p.box_n;
+    // The MMA always reads a 128-row A tile; when fewer rows are loaded the rest of that window is
+    // whatever follows in shared memory (rows that no output uses), so keep the window in bounds.
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES + (A_TILE_BYTES - A_BYTES));
     // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
     const uint32_t bar_full = smem_u32(bars);
-    const uint32_t bar_empty = bar_full + 8 * STAGES;
-    const uint32_t bar_tfull = bar_empty + 8 * STAGES;
+    const uint32_t bar_empty = bar_full + 8 * MAX_STAGES;
+    const uint32_t bar_tfull = bar_empty + 8 * MAX_STAGES;
     const uint32_t bar_tempty = bar_tfull + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* is_last = reinterpret_cast<int*>(tmem_slot + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_units = p.n_mtiles * p.n_chunks;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -249,8 +268,10 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const Unit un = decode_unit(p, u);
+            UnitIter it(p);
+            Unit un;
+            const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2;
+            while (ok && it.next(p, un)) {
                 for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES) {
                     const int nb = min(MAX_BOXES, un.box_end - b0);
                     for (int kb = 0; kb < p.num_kb; ++kb) {
@@ -260,7 +281,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                         const uint32_t full = bar_full + 8 * stage;
                         const uint32_t sa = tiles + stage * STAGE_BYTES;
-                        mbar_expect_tx(full, (uint32_t)(A_BYTES + nb * BOX_BYTES));
+                        mbar_expect_tx(full, a_box_bytes + (uint32_t)(nb * BOX_BYTES));
                         tma_load_2d(sa, &tmA, kb * BLOCK_K, un.m_tile * BLOCK_M, full);
                         for (int j = 0; j < nb; ++j)
                             tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, kb * BLOCK_K, (b0 + j) * BOX_N, full);
@@ -294,8 +315,9 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t phase = 0;
             uint32_t tile = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const Unit un = decode_unit(p, u);
+            UnitIter it(p);
+            Unit un;
+            while (ok && it.next(p, un)) {
                 for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
                     const int nb = min(MAX_BOXES, un.box_end - b0);
                     const uint32_t as = tile & 1u, aphase = (tile >> 1) & 1u;
@@ -335,20 +357,23 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
         uint32_t tile = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-            const Unit un = decode_unit(p, u);
+        UnitIter it(p);
+        Unit un;
+        while (ok && it.next(p, un)) {
             const int row = un.m_tile * BLOCK_M + row_in_tile;
             // running reduction of this row over the unit's columns
             float best_v = -INFINITY;
             int best_i = 0x7FFFFFFF;
-            float tv[MODE == MODE_TOPK ? kMaxKTab : 1];
-            int ti[MODE == MODE_TOPK ? kMaxKTab : 1];
-            float thr = -INFINITY;
-            if (MODE == MODE_TOPK) {
-                for (int j = 0; j < p.k_tab; ++j) {
-                    tv[j] = -INFINITY;
-                    ti[j] = 0x7FFFFFFF;
-                }
+            // Sorted list, value descending, statically indexed so it stays in registers.  The k_tab live
+            // entries sit at the bottom [KT - k_tab, KT); the slots above hold +inf, which nothing beats,
+            // so the running threshold is always the last slot.
+            float tv[KT];
+            int ti[KT];
+            const int k_off = KT - p.k_tab;
+#pragma unroll
+            for (int j = 0; j < KT; ++j) {
+                tv[j] = j < k_off ? INFINITY : -INFINITY;
+                ti[j] = 0x7FFFFFFF;
             }
             for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
                 const int nb = min(MAX_BOXES, un.box_end - b0);
@@ -360,8 +385,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 tc_fence_after();
                 const int col0 = b0 * BOX_N;
                 const int n_valid = min(nb * BOX_N, p.V - col0);
-                for (int c = 0; c < nb; ++c) {
-                    if (c * 32 >= n_valid) break;
+                for (int c = 0; c * 32 < n_valid; ++c) {
                     uint32_t r[32];
                     __syncwarp();
                     tmem_ld32(lane_base + as * ACC_COLS + c * 32, r);
@@ -381,16 +405,24 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             const float v = __uint_as_float(r[j]);
-                            if (j < lim && v > thr) {
-                                int pos = p.k_tab - 1;
-                                while (pos > 0 && v > tv[pos - 1]) {
-                                    tv[pos] = tv[pos - 1];
-                                    ti[pos] = ti[pos - 1];
-                                    --pos;
+                            if (j < lim && v > tv[KT - 1]) {
+                                // branch-free insertion from the bottom up: slot q takes its upper
+                                // neighbour if v also beats that one, else v itself; strict compares
+                                // keep earlier (lower) token ids ahead of equal values
+                                const int c_id = cbase + j;
+#pragma unroll
+                                for (int q = KT - 1; q > 0; --q) {
+                                    const bool up = v > tv[q - 1];
+                                    const bool wr = v > tv[q];
+                                    const float nv = up ? tv[q - 1] : v;
+                                    const int ni = up ? ti[q - 1] : c_id;
+                                    tv[q] = wr ? nv : tv[q];
+                                    ti[q] = wr ? ni : ti[q];
                                 }
-                                tv[pos] = v;
-                                ti[pos] = cbase + j;
-                                thr = tv[p.k_tab - 1];
+                                if (v > tv[0]) {
+                                    tv[0] = v;
+                                    ti[0] = c_id;
+                                }
                             }
                         }
                     } else {
@@ -414,10 +446,12 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     atomicMax(p.keys + row, key);
                 } else if (MODE == MODE_TOPK) {
                     const size_t base = ((size_t)un.chunk * p.a_rows + row) * p.k_tab;
-                    for (int j = 0; j < p.k_tab; ++j) {
-                        p.part_val[base + j] = tv[j];
-                        p.part_idx[base + j] = ti[j];
-                    }
+#pragma unroll
+                    for (int j = 0; j < KT; ++j)
+                        if (j >= k_off) {
+                            p.part_val[base + j - k_off] = tv[j];
+                            p.part_idx[base + j - k_off] = ti[j];
+                        }
                 }
             }
         }
@@ -503,68 +537,105 @@ __global__ void extend_table_kernel(const int32_t* __restrict__ tab, int V, int 
 
 // ------------------------------------------------------------------------------------------ host: unit shapes
 struct Shape {
-    int n_chunks, align, group, grid;
+    int box_n, box_idx, group, n_groups, n_slots, n_chunks, grid;
+    int a_box_rows, a_bytes, stage_bytes, stages, smem;
 };
 
-// Static-striding makespan of a candidate split, in boxes (a tile costs its boxes plus a fixed overhead).
-static double makespan(int n_mtiles, int n_boxes, int n_chunks, int align, int group, int grid) {
-    std::vector<double> load((size_t)grid, 0.0);
-    const long long n_al = (n_boxes + align - 1) / align;
-    const int per_group = group * n_chunks;
-    const int n_units = n_mtiles * n_chunks;
-    for (int u = 0; u < n_units; ++u) {
-        const int mg = u / per_group;
-        const int g = std::min(group, n_mtiles - mg * group);
-        const int chunk = (u - mg * per_group) / g;
-        const int b0 = (int)((long long)chunk * n_al / n_chunks) * align;
-        const int b1 = std::min(n_boxes, (int)((long long)(chunk + 1) * n_al / n_chunks) * align);
-        const int boxes = b1 - b0;
-        const int tiles = (boxes + MAX_BOXES - 1) / MAX_BOXES;
-        load[(size_t)(u % grid)] += boxes + 0.75 * tiles + 0.25;
-    }
-    double mx = 0;
-    for (double v : load) mx = std::max(mx, v);
-    return mx;
+// Derives the shared-memory geometry from (box_n, group, n_chunks, grid).
+static void finish_shape(Shape& sh, int a_rows, int V) {
+    const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
+    sh.box_idx = sh.box_n == 16 ? 0 : sh.box_n == 32 ? 1 : sh.box_n == 64 ? 2 : sh.box_n == 128 ? 3 : 4;
+    sh.n_groups = (n_mtiles + sh.group - 1) / sh.group;
+    sh.n_slots = sh.grid / sh.group;
+    const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
+    const int chunk_max = (n_boxes + sh.n_chunks - 1) / sh.n_chunks;
+    const int nb_max = std::min(TILE_N / sh.box_n, chunk_max);
+    sh.a_box_rows = n_mtiles == 1 ? std::min(BLOCK_M, (a_rows + 7) / 8 * 8) : BLOCK_M;
+    sh.a_bytes = (sh.a_box_rows * BLOCK_K * 2 + 1023) / 1024 * 1024;
+    sh.stage_bytes = sh.a_bytes + (nb_max * sh.box_n * BLOCK_K * 2 + 1023) / 1024 * 1024;
+    const int pad = A_TILE_BYTES - sh.a_bytes;
+    sh.stages = std::min(MAX_STAGES, (SMEM_LIMIT - SMEM_MISC - pad) / sh.stage_bytes);
+    sh.smem = sh.stages * sh.stage_bytes + pad + SMEM_MISC;
 }
 
-static Shape choose_shape(int n_mtiles, int n_boxes, int sms, int max_chunks) {
-    Shape best{1, 1, 1, 1};
-    double best_cost = 1e300;
-    const int group = std::min(n_mtiles, 8);
-    const int n_tiles = (n_boxes + MAX_BOXES - 1) / MAX_BOXES;
-    for (int align = 1; align <= MAX_BOXES; align += MAX_BOXES - 1) {
-        const int limit = std::min(max_chunks, align == 1 ? n_boxes : n_tiles);
-        for (int c = 1; c <= limit; ++c) {
-            // fine-grained (align 1) splits only make sense while a chunk is at most one tile
-            if (align == 1 && (n_boxes + c - 1) / c > MAX_BOXES && c > 1) continue;
-            const int units = n_mtiles * c;
-            const int grid = std::min(units, sms);
-            const double cost = makespan(n_mtiles, n_boxes, c, align, group, grid) * (1.0 + 1e-4 * c);
-            if (cost < best_cost) {
-                best_cost = cost;
-                best = Shape{c, align, group, grid};
+// Unit shapes.  One m-tile (memory-bound): every SM streams its own slice of W once, in 32-row
+// boxes so slices balance to within one box.  Several m-tiles (tensor-bound): `group` m-tiles
+// share each W chunk, W is loaded in large boxes (few TMA issues per k-block), and the chunk
+// count is a multiple of the slots so that every slot sweeps the same number of chunks.
+static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks) {
+    const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
+    Shape sh{};
+    if (n_mtiles == 1) {
+        sh.box_n = 32;
+        sh.group = 1;
+        sh.n_chunks = (int)std::min<size_t>((size_t)std::min(sms, (V + 31) / 32), max_chunks);
+        sh.grid = sh.n_chunks;
+    } else {
+        sh.box_n = 64;
+        // the largest group up to 8 that leaves the fewest SMs idle, counting a ragged last m-group
+        double best = -1.0;
+        for (int g = std::min(8, n_mtiles); g >= 1; --g) {
+            const int slots = sms / g, groups = (n_mtiles + g - 1) / g;
+            const double busy = (double)n_mtiles / (groups * g) * (double)(slots * g) / sms * (1.0 - 0.01 * (8 - g));
+            if (busy > best + 1e-9) {
+                best = busy;
+                sh.group = g;
             }
         }
+        const int slots = sms / sh.group;
+        const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
+        sh.n_chunks = (int)std::min<size_t>((size_t)std::min(slots, n_boxes), max_chunks);
+        sh.grid = sh.group * std::min(slots, sh.n_chunks);
     }
-    return best;
+    finish_shape(sh, a_rows, V);
+    return sh;
 }
 
-static Shape cached_shape(spec_ctx* ctx, int n_mtiles, int n_boxes, int max_chunks) {
-    static std::map<std::tuple<int, int, int, int>, Shape> cache;
-    const auto key = std::make_tuple(n_mtiles, n_boxes, ctx->num_sms, max_chunks);
+static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks) {
+    // Tuning aid: NGRAM_SPEC_SHAPE="box,group,chunks" overrides the choice (values are clamped).
+    if (const char* ov = getenv("NGRAM_SPEC_SHAPE")) {
+        int box = 32, g = 1, c = 1;
+        if (sscanf(ov, "%d,%d,%d", &box, &g, &c) == 3 && (box == 16 || box == 32 || box == 64 || box == 128 || box == 256)) {
+            const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
+            Shape s{};
+            s.box_n = box;
+            s.group = std::max(1, std::min(std::min(g, n_mtiles), ctx->num_sms));
+            const int n_boxes = (ctx->V + box - 1) / box;
+            s.n_chunks = (int)std::max<size_t>(1, std::min<size_t>(std::min<size_t>((size_t)std::max(c, 1), (size_t)n_boxes), max_chunks));
+            s.grid = s.group * std::min(ctx->num_sms / s.group, s.n_chunks);
+            finish_shape(s, a_rows, ctx->V);
+            return s;
+        }
+    }
+    static std::map<std::tuple<int, int, int, int, size_t>, Shape> cache;
+    const auto key = std::make_tuple(a_rows, ctx->V, ctx->d, ctx->num_sms, max_chunks);
     auto it = cache.find(key);
     if (it != cache.end()) return it->second;
-    Shape s = choose_shape(n_mtiles, n_boxes, ctx->num_sms, max_chunks);
+    Shape s = choose_shape(a_rows, ctx->V, ctx->num_sms, max_chunks);
     cache[key] = s;
+    if (getenv("NGRAM_SPEC_TRACE"))
+        fprintf(stderr, "[ngram_spec] rows=%d V=%d d=%d: box=%d group=%d slots=%d chunks=%d grid=%d a_box=%d stages=%d stage=%dB smem=%dB\n",
+                a_rows, ctx->V, ctx->d, s.box_n, s.group, s.n_slots, s.n_chunks, s.grid, s.a_box_rows, s.stages, s.stage_bytes, s.smem);
     return s;
 }
 
-template <int MODE>
+// Tensor map of the unembedding for the shape's box size (encoded once per context).
+static int w_map(spec_ctx* ctx, const Shape& sh, const CUtensorMap** out) {
+    if (!ctx->tm_w_ready[sh.box_idx]) {
+        int rc = make_tensor_map(ctx, &ctx->tm_w[sh.box_idx], ctx->unembed, ctx->V, ctx->d, sh.box_n);
+        if (rc) return rc;
+        ctx->tm_w_ready[sh.box_idx] = true;
+    }
+    *out = &ctx->tm_w[sh.box_idx];
+    return SPEC_OK;
+}
+
+template <int MODE, int KT>
 static int set_smem_attr(spec_ctx* ctx) {
     static bool done[64] = {false};
     bool& d = done[ctx->device & 63];
     if (d) return SPEC_OK;
-    int rc = check_cuda(ctx, cudaFuncSetAttribute(head_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM),
+    int rc = check_cuda(ctx, cudaFuncSetAttribute(head_gemm_kernel<MODE, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT),
                         "head gemm: cudaFuncSetAttribute");
     if (rc == SPEC_OK) d = true;
     return rc;
@@ -575,10 +646,16 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.V = ctx->V;
     p.num_kb = (ctx->d + BLOCK_K - 1) / BLOCK_K;
     p.n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
-    p.n_boxes = (ctx->V + BOX_N - 1) / BOX_N;
+    p.box_n = sh.box_n;
+    p.n_boxes = (ctx->V + sh.box_n - 1) / sh.box_n;
     p.n_chunks = sh.n_chunks;
-    p.align = sh.align;
     p.group = sh.group;
+    p.n_groups = sh.n_groups;
+    p.n_slots = sh.n_slots;
+    p.a_box_rows = sh.a_box_rows;
+    p.a_bytes = sh.a_bytes;
+    p.stage_bytes = sh.stage_bytes;
+    p.stages = sh.stages;
     p.keys = ctx->d_keys;
     p.ticket = ctx->d_ticket;
     p.argmax = nullptr;
@@ -591,48 +668,51 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
 }
 
 int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st) {
-    int rc = set_smem_attr<MODE_ARGMAX>(ctx);
+    int rc = set_smem_attr<MODE_ARGMAX, 1>(ctx);
     if (rc) return rc;
+    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20);
+    const CUtensorMap* tmW;
+    if ((rc = w_map(ctx, sh, &tmW))) return rc;
     CUtensorMap tmA;
-    if ((rc = make_tensor_map(ctx, &tmA, d_hidden, M, ctx->d, BLOCK_M))) return rc;
-    const int n_mtiles = (M + BLOCK_M - 1) / BLOCK_M, n_boxes = (ctx->V + BOX_N - 1) / BOX_N;
-    const Shape sh = cached_shape(ctx, n_mtiles, n_boxes, 256);
+    if ((rc = make_tensor_map(ctx, &tmA, d_hidden, M, ctx->d, sh.a_box_rows))) return rc;
     GemmParams p;
     fill_common(ctx, p, M, sh);
     p.argmax = d_argmax;
     p.maxv = d_max;
-    head_gemm_kernel<MODE_ARGMAX><<<sh.grid, GEMM_THREADS, GEMM_SMEM, st>>>(tmA, ctx->tm_unembed, p);
+    head_gemm_kernel<MODE_ARGMAX, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, cudaGetLastError(), "verify_lmhead_argmax launch");
 }
 
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st) {
-    int rc = set_smem_attr<MODE_STORE>(ctx);
+    int rc = set_smem_attr<MODE_STORE, 1>(ctx);
     if (rc) return rc;
+    const Shape sh = cached_shape(ctx, m, (size_t)1 << 20);
+    const CUtensorMap* tmW;
+    if ((rc = w_map(ctx, sh, &tmW))) return rc;
     CUtensorMap tmA;
-    if ((rc = make_tensor_map(ctx, &tmA, d_rows, m, ctx->d, BLOCK_M))) return rc;
-    const int n_mtiles = (m + BLOCK_M - 1) / BLOCK_M, n_boxes = (ctx->V + BOX_N - 1) / BOX_N;
-    const Shape sh = cached_shape(ctx, n_mtiles, n_boxes, 256);
+    if ((rc = make_tensor_map(ctx, &tmA, d_rows, m, ctx->d, sh.a_box_rows))) return rc;
     GemmParams p;
     fill_common(ctx, p, m, sh);
     p.logits = d_logits;
-    head_gemm_kernel<MODE_STORE><<<sh.grid, GEMM_THREADS, GEMM_SMEM, st>>>(tmA, ctx->tm_unembed, p);
+    head_gemm_kernel<MODE_STORE, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, cudaGetLastError(), "spec_debug_logits launch");
 }
 
 int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
                  int32_t* d_ext, cudaStream_t st) {
-    int rc = set_smem_attr<MODE_TOPK>(ctx);
+    const int kt = k_tab <= 8 ? 8 : (k_tab <= 16 ? 16 : 32);
+    int rc = kt == 8 ? set_smem_attr<MODE_TOPK, 8>(ctx) : (kt == 16 ? set_smem_attr<MODE_TOPK, 16>(ctx) : set_smem_attr<MODE_TOPK, 32>(ctx));
     if (rc) return rc;
     const int V = ctx->V;
-    CUtensorMap tmA;
-    if ((rc = make_tensor_map(ctx, &tmA, d_rows, V, ctx->d, BLOCK_M))) return rc;
-    const int n_mtiles = (V + BLOCK_M - 1) / BLOCK_M, n_boxes = (V + BOX_N - 1) / BOX_N;
     // partial lists cost 8 bytes per entry and chunk: keep them under 256 MB
     int max_chunks = (int)std::max<long long>(1, (256ll << 20) / ((long long)V * k_tab * 8));
-    max_chunks = std::min(max_chunks, 64);
-    const Shape sh = cached_shape(ctx, n_mtiles, n_boxes, max_chunks);
+    const Shape sh = cached_shape(ctx, V, (size_t)max_chunks);
+    const CUtensorMap* tmW;
+    if ((rc = w_map(ctx, sh, &tmW))) return rc;
+    CUtensorMap tmA;
+    if ((rc = make_tensor_map(ctx, &tmA, d_rows, V, ctx->d, sh.a_box_rows))) return rc;
     const size_t need = (size_t)sh.n_chunks * V * k_tab;
     if (need > ctx->part_capacity) {
         cudaStreamSynchronize(st);
@@ -650,7 +730,12 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
     p.k_tab = k_tab;
     p.part_val = ctx->d_part_val;
     p.part_idx = ctx->d_part_idx;
-    head_gemm_kernel<MODE_TOPK><<<sh.grid, GEMM_THREADS, GEMM_SMEM, st>>>(tmA, ctx->tm_unembed, p);
+    if (kt == 8)
+        head_gemm_kernel<MODE_TOPK, 8><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
+    else if (kt == 16)
+        head_gemm_kernel<MODE_TOPK, 16><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
+    else
+        head_gemm_kernel<MODE_TOPK, 32><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
     if ((rc = check_cuda(ctx, cudaGetLastError(), "build_model_ngram_tables launch"))) return rc;
     merge_topk_kernel<<<(V + 127) / 128, 128, 0, st>>>(ctx->d_part_val, ctx->d_part_idx, sh.n_chunks, V, k_tab, d_tab_idx,
                                                       d_tab_val);
@@ -733,8 +818,8 @@ extern "C" int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d,
     tmp.d_ticket = reinterpret_cast<unsigned int*>(nd.scratch + SPEC_NOALLOC_MAX_ROWS);
     tmp.d_status = reinterpret_cast<int*>(nd.scratch + SPEC_NOALLOC_MAX_ROWS + 1);
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = make_tensor_map(&tmp, &tmp.tm_unembed, d_unembed, V, d, BOX_N);
-    if (rc == SPEC_OK) {
+    int rc = SPEC_OK;
+    {
         // The scratch keeps whatever the previous call left: the keys of this call's rows, the ticket and
         // the status word must start at zero.  Outputs start at -1 so an expired wait cannot pass for a result.
         e = cudaMemsetAsync(nd.scratch, 0, sizeof(unsigned long long) * (size_t)M, st);
