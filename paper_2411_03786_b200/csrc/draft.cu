@@ -34,6 +34,8 @@ struct DraftParams {
 };
 
 constexpr int kMaxPasses = 1024;
+constexpr int kRankMax = 512;                          // groups ranked by counting (all threads) up to here
+constexpr int kMaxCand = kMaxNQ * kMaxB + kMaxKTab;    // candidate rows before duplicates are dropped
 
 __device__ __forceinline__ uint32_t fmix32(uint32_t h) {
     h ^= h >> 16;
@@ -55,9 +57,13 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 
 struct DraftSmem {
     unsigned long long run_key[kMaxNQ][kMaxB];  // per query length: ranked (count << 32 | start) keys
-    int32_t out[kMaxB][kMaxW];
-    int32_t out_src[kMaxB];
-    int32_t out_cnt[kMaxB];
+    unsigned long long gkey[kRankMax];          // (query index << 60 | count << 32 | start) per group
+    int32_t cand_src[kMaxCand];
+    int32_t cand_cnt[kMaxCand];
+    int32_t cand_keep[kMaxCand];
+    int32_t row_of[kMaxB];                      // candidate that became draft row b
+    int cand_off[kMaxNQ + 2];
+    int n_cnt[kMaxNQ];
     int32_t chain[kMaxKTab][kMaxW];
     int chain_ok[kMaxKTab];
     int n_run[kMaxNQ];
@@ -109,7 +115,7 @@ __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int 
     sm->overflow = 1;
 }
 
-__global__ void __launch_bounds__(1024) draft_kernel(const DraftParams P) {
+__global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DraftSmem* sm = reinterpret_cast<DraftSmem*>(smem_raw);
     int* rep = reinterpret_cast<int*>(smem_raw + ((sizeof(DraftSmem) + 15) & ~size_t(15)));
@@ -229,8 +235,32 @@ __global__ void __launch_bounds__(1024) draft_kernel(const DraftParams P) {
                 overflowed = true;
                 break;
             }
-            // rank this pass's groups together with the winners of earlier passes: warp qi
-            if (warp < P.n_q) {
+            if (R == 1 && sm->n_groups <= kRankMax) {
+                // Few groups (the usual case): every thread ranks groups by counting the groups of the same
+                // query length with a larger (count, start) key; rank r < topk lands in slot r.
+                const int n_groups = sm->n_groups;
+                if (tid < kMaxNQ) sm->n_cnt[tid] = 0;
+                for (int g = tid; g < n_groups; g += nthr) {
+                    const int slot = grp_slot[g];
+                    const unsigned long long qi = (unsigned long long)(rep[slot] >> 28);
+                    sm->gkey[g] = (qi << 60) | ((unsigned long long)(uint32_t)cnt[slot] << 32) | (uint32_t)last[slot];
+                }
+                __syncthreads();
+                for (int g = tid; g < n_groups; g += nthr) {
+                    const unsigned long long mine = sm->gkey[g];
+                    int rank = 0;
+                    for (int o = 0; o < n_groups; ++o) {
+                        const unsigned long long other = sm->gkey[o];
+                        rank += ((other >> 60) == (mine >> 60) && other > mine) ? 1 : 0;
+                    }
+                    const int qi = (int)(mine >> 60);
+                    atomicAdd(&sm->n_cnt[qi], 1);
+                    if (rank < P.topk) sm->run_key[qi][rank] = mine & 0x0FFFFFFFFFFFFFFFull;
+                }
+                __syncthreads();
+                if (tid < kMaxNQ) sm->n_run[tid] = min(P.topk, sm->n_cnt[tid]);
+            } else if (warp < P.n_q) {
+                // rank this pass's groups together with the winners of earlier passes: warp qi
                 const int qi = warp;
                 const int n_groups = sm->n_groups;
                 const int n_old = sm->n_run[qi];
@@ -277,54 +307,88 @@ __global__ void __launch_bounds__(1024) draft_kernel(const DraftParams P) {
     }
     __syncthreads();
 
-    // ---- mixed allocation: context rows in query order, then model rows by rank; drop duplicates
-    if (warp == 0) {
-        int n = 0;
-        const bool dedup = (P.flags & SPEC_FLAG_DEDUP) != 0;
-        const int n_model = (P.flags & SPEC_FLAG_MODEL_FILL) ? P.k_tab : 0;
-        const int n_lists = P.n_q + 1;
-        for (int li = 0; li < n_lists && n < P.B; ++li) {
-            const bool model = (li == P.n_q);
-            const int n_cand = model ? n_model : sm->n_run[li];
-            for (int r = 0; r < n_cand && n < P.B; ++r) {
-                int tok = -1, count = 0;
-                if (model) {
-                    if (!sm->chain_ok[r]) continue;
-                    if (lane < w) tok = sm->chain[r][lane];
-                } else {
-                    const unsigned long long key = sm->run_key[li][r];
-                    const int p = (int)(uint32_t)key;
-                    count = (int)(key >> 32);
-                    if (lane < w) tok = h[p + lane];
-                }
-                bool dup = false;
-                if (dedup) {
-                    for (int b = 0; b < n && !dup; ++b) {
-                        const bool eq = (lane < w) ? (sm->out[b][lane] == tok) : true;
-                        dup = __all_sync(0xffffffffu, eq);
-                    }
-                }
-                if (dup) continue;
-                if (lane < w) sm->out[n][lane] = tok;
-                if (lane == 0) {
-                    sm->out_src[n] = model ? 0 : P.qs[li];
-                    sm->out_cnt[n] = count;
-                }
-                __syncwarp();
-                ++n;
-            }
+    // ---- mixed allocation: context rows in query order, then model rows by rank; drop duplicates.
+    // Candidate rows are gathered side by side, a row is a duplicate if any earlier candidate equals
+    // it (equality is transitive, so this is the same as comparing with the rows already taken),
+    // and the first B survivors become the drafts.
+    const bool dedup = (P.flags & SPEC_FLAG_DEDUP) != 0;
+    if (tid == 0) {
+        int off = 0;
+        for (int li = 0; li < P.n_q; ++li) {
+            sm->cand_off[li] = off;
+            off += sm->n_run[li];
         }
-        if (lane == 0) sm->n_out = n;
+        sm->cand_off[P.n_q] = off;
+        off += (P.flags & SPEC_FLAG_MODEL_FILL) ? P.k_tab : 0;
+        sm->cand_off[P.n_q + 1] = off;
+    }
+    __syncthreads();
+    int32_t* cand = rep;  // the hash table is no longer needed: [n_cand][w] token rows
+    const int n_cand = sm->cand_off[P.n_q + 1];
+    for (int i = tid; i < n_cand * w; i += nthr) {
+        const int ci = i / w, t = i - ci * w;
+        int li = 0;
+        while (ci >= sm->cand_off[li + 1]) ++li;
+        const int r = ci - sm->cand_off[li];
+        int tok, keep = 1, src = 0, count = 0;
+        if (li == P.n_q) {
+            keep = sm->chain_ok[r];
+            tok = keep ? sm->chain[r][t] : -1;
+        } else {
+            const unsigned long long key = sm->run_key[li][r];
+            tok = h[(int)(uint32_t)key + t];
+            src = P.qs[li];
+            count = (int)(key >> 32);
+        }
+        cand[i] = tok;
+        if (t == 0) {
+            sm->cand_src[ci] = src;
+            sm->cand_cnt[ci] = count;
+            sm->cand_keep[ci] = keep;
+        }
+    }
+    __syncthreads();
+    if (dedup) {
+        int drop[(kMaxCand + 127) / 128];  // decisions first, writes after: cand_keep is read by others (>= 128 threads)
+        int n_mine = 0;
+        for (int ci = tid; ci < n_cand; ci += nthr, ++n_mine) {
+            bool dup = false;
+            if (sm->cand_keep[ci])
+                for (int j = 0; j < ci && !dup; ++j) {
+                    if (!sm->cand_keep[j]) continue;  // an invalid model row
+                    bool same = true;
+                    for (int t = 0; t < w && same; ++t) same = cand[j * w + t] == cand[ci * w + t];
+                    dup = same;
+                }
+            drop[n_mine] = dup ? 1 : 0;
+        }
+        __syncthreads();
+        n_mine = 0;
+        for (int ci = tid; ci < n_cand; ci += nthr, ++n_mine)
+            if (drop[n_mine]) sm->cand_keep[ci] = 0;
+        __syncthreads();
+    }
+    if (warp == 0) {
+        int base = 0;
+        for (int c0 = 0; c0 < n_cand; c0 += 32) {
+            const int ci = c0 + lane;
+            const bool k = ci < n_cand && sm->cand_keep[ci] != 0;
+            const unsigned mask = __ballot_sync(0xffffffffu, k);
+            const int pos = base + __popc(mask & ((1u << lane) - 1u));
+            if (k && pos < P.B) sm->row_of[pos] = ci;
+            base += __popc(mask);
+        }
+        if (lane == 0) sm->n_out = min(base, P.B);
     }
     __syncthreads();
     const int n = sm->n_out;
     for (int i = tid; i < P.B * w; i += nthr) {
         const int b = i / w, t = i - b * w;
-        P.drafts[(size_t)s * P.B * w + i] = (b < n) ? sm->out[b][t] : -1;
+        P.drafts[(size_t)s * P.B * w + i] = (b < n) ? cand[sm->row_of[b] * w + t] : -1;
     }
     for (int b = tid; b < P.B; b += nthr) {
-        if (P.src) P.src[(size_t)s * P.B + b] = (b < n) ? sm->out_src[b] : -1;
-        if (P.counts) P.counts[(size_t)s * P.B + b] = (b < n) ? sm->out_cnt[b] : 0;
+        if (P.src) P.src[(size_t)s * P.B + b] = (b < n) ? sm->cand_src[sm->row_of[b]] : -1;
+        if (P.counts) P.counts[(size_t)s * P.B + b] = (b < n) ? sm->cand_cnt[sm->row_of[b]] : 0;
     }
     if (tid == 0) P.ndrafts[s] = n;
 }
@@ -362,8 +426,9 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.slots = slots;
     P.max_groups = slots / 2;
     const int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);
-    const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + (size_t)slots * 3 * sizeof(int) +
-                        (size_t)P.max_groups * sizeof(int);
+    const size_t table_bytes = (size_t)slots * 3 * sizeof(int) + (size_t)P.max_groups * sizeof(int);
+    const size_t cand_bytes = (size_t)(n_q * topk + kMaxKTab) * w * sizeof(int32_t);  // aliases the table
+    const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + (table_bytes > cand_bytes ? table_bytes : cand_bytes);
     static bool attr_set[64] = {false};
     bool& attr_done = attr_set[ctx->device & 63];
     if (!attr_done) {
