@@ -312,15 +312,9 @@ def main():
     d2h = h_acc.numel() * 4 + h_com.numel() * 4
 
     # ---- max over ranks, totals over ranks
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms, verify_ms, verify_alone_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, verify_ms, verify_alone_ms = (float(x) for x in t)
-        a = torch.tensor([acc_mean], device=dev, dtype=torch.float64)
-        dist.all_reduce(a, op=dist.ReduceOp.SUM)
-        acc_total = float(a[0])
-    else:
-        acc_total = acc_mean
+    from paper_2411_03786_b200.multigpu import reduce_max_sum
+    (total_ms, e2e_ms, verify_ms, verify_alone_ms), (acc_total,) = reduce_max_sum(
+        [total_ms, e2e_ms, verify_ms, verify_alone_ms], [acc_mean], device=dev)
     ms_per_step = total_ms / args.steps
     value = acc_total / (ms_per_step / 1e3)
     e2e_value = acc_total / (e2e_ms / args.steps / 1e3)
@@ -355,7 +349,7 @@ def main():
                 "phase_ms": {"draft": draft_ms, "verify": verify_ms, "accept": accept_ms},
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms / args.steps},
-                "gpu_launches": int(launches), "launch_mode": "eager" if graph is None else "cuda_graph_replay", "roofline": roof, "table_build": table, "cpu_baseline": cpu,
+                "gpu_launches": int(launches) * world, "launch_mode": "eager" if graph is None else "cuda_graph_replay", "roofline": roof, "table_build": table, "cpu_baseline": cpu,
                 "clocks": clk.summary(), "status_bits": status, "copied_fraction": copied}
         print(json.dumps(line))
     ctx.close()
