@@ -136,6 +136,61 @@ def oracle_step_time(c, hist, lens, T, H_bits, W_bits, budget_s, min_steps=1, ma
     return total / steps, accepted / steps, threads, sample, rows is not None
 
 
+def scaled_streams(ctx, torch, dev, c, pk):
+    """Streaming rates of the integer kernels on batches large enough to measure bandwidth (at the
+    benchmark sizes they move a few KB and are launch-latency-bound)."""
+    out = {}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    for S, L, reps in ((4096, 2048, 20), (512, 131072, 5)):
+        base, lens_b, _ = synth.zipf_histories(32, L, c["V"], c["zipf"], 0.3, seed=77, cap=L + 64, name="scaled")
+        hist = torch.from_numpy(np.tile(base, (S // 32, 1))).to(dev)
+        lens = torch.from_numpy(np.tile(lens_b, S // 32)).to(dev)
+        B, w, topk, qs = 16, 8, 4, (3, 2, 1)
+        bufs = (torch.empty((S, B, w), dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+                torch.empty((S, B), dtype=torch.int32, device=dev), torch.empty((S, B), dtype=torch.int32, device=dev))
+        ms = timed(lambda: ctx.draft_context_ngrams(hist, lens, qs, topk, B, w, out=bufs), reps)
+        by = 4.0 * S * L + 4.0 * S * B * (w + 2) + 8.0 * S
+        out[f"draft_S{S}_L{L}"] = {"ms": ms, "GB/s": by / ms / 1e6, "frac_of_hbm": by / ms / 1e6 / pk["hbm"], "bytes": by,
+                                   "l2": "larger than L2" if by > 126e6 else "L2-resident"}
+        del hist, lens, bufs
+    S, B, w = 65536, 64, 10
+    g = torch.Generator(device=dev).manual_seed(3)
+    drafts = torch.randint(0, 4, (S, B, w), device=dev, dtype=torch.int32, generator=g)
+    P = torch.randint(0, 4, (S, B, w + 1), device=dev, dtype=torch.int32, generator=g)
+    nd = torch.full((S,), B, dtype=torch.int32, device=dev)
+    cap = 64
+    hist = torch.zeros((S, cap), dtype=torch.int32, device=dev)
+    lens0 = torch.full((S,), 8, dtype=torch.int32, device=dev)
+    lens = lens0.clone()
+    bufs = (torch.empty(S, dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+            torch.empty((S, w + 1), dtype=torch.int32, device=dev))
+
+    def acc():
+        lens.copy_(lens0)
+        ctx.accept_and_commit(drafts, nd, P, hist, lens, out=bufs)
+
+    ms = timed(acc, 10)
+    # early exit reads only the first sector of most rows: count the bytes of every 32-byte sector touched at
+    # least once, i.e. the first sector of each draft row and of each prediction row, plus the outputs
+    by_full = 4.0 * S * B * (2 * w + 1) + 4.0 * S * (w + 4)
+    out[f"accept_S{S}_B{B}_w{w}"] = {"ms": ms, "GB/s_if_all_bytes_read": by_full / ms / 1e6, "bytes_all": by_full,
+                                    "note": "prefix comparison stops at the first mismatch, so fewer bytes are needed"}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -145,6 +200,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU work for the oracle baseline")
     ap.add_argument("--no-table", action="store_true", help="skip timing the one-off table build")
+    ap.add_argument("--scaled", action="store_true", help="also time draft/accept on bandwidth-sized batches")
     ap.add_argument("--no-graph", action="store_true", help="launch the step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -334,6 +390,7 @@ def main():
                  "ms_per_launch": verify_alone_ms, "timing": "CUDA events around back-to-back launches on the launching stream", "algorithmic_bytes": bytes_alg, "flops": flops,
                  "peak_source": pk["source"] + (" sustained" if roof["bound"] == "tensor" else " copy")})
 
+    scaled = scaled_streams(ctx, torch, dev, c, pk) if (args.scaled and rank == 0) else None
     line = None
     if rank == 0:
         cpu = {}
@@ -351,6 +408,8 @@ def main():
                         "ms_per_step": e2e_ms / args.steps},
                 "gpu_launches": int(launches) * world, "launch_mode": "eager" if graph is None else "cuda_graph_replay", "roofline": roof, "table_build": table, "cpu_baseline": cpu,
                 "clocks": clk.summary(), "status_bits": status, "copied_fraction": copied}
+        if scaled:
+            line["scaled_streams"] = scaled
         print(json.dumps(line))
     ctx.close()
     if dist is not None:
