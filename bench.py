@@ -343,7 +343,7 @@ def main():
     h_acc, h_com = torch.empty(S, dtype=torch.int32).pin_memory(), torch.empty((S, w + 1), dtype=torch.int32).pin_memory()
     d_hist2, d_H2 = torch.empty_like(hist), torch.empty_like(dH.view(torch.int16))
 
-    def e2e_step():
+    def e2e_body():
         d_hist2.copy_(h_hist, non_blocking=True)
         lens.copy_(h_lens, non_blocking=True)
         d_H2.copy_(h_H, non_blocking=True)
@@ -352,7 +352,23 @@ def main():
         ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), d_hist2, lens, out=out_a)
         h_acc.copy_(out_a[0], non_blocking=True)
         h_com.copy_(out_a[2], non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+
+    e2e_graph = None
+    if graph is not None:
+        with torch.cuda.stream(side):
+            e2e_body()
+        torch.cuda.synchronize()
+        e2e_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(e2e_graph, stream=side):
+            e2e_body()
+
+    def e2e_step():
+        # host -> device copies, the three kernels and the device -> host read-back, then wait for the result
+        if e2e_graph is not None:
+            e2e_graph.replay()
+        else:
+            e2e_body()
+        torch.cuda.synchronize()
 
     for _ in range(3):
         e2e_step()
