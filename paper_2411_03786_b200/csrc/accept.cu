@@ -13,6 +13,8 @@ __global__ void __launch_bounds__(128) accept_commit_kernel(
     int* __restrict__ status) {
     const int lane = threadIdx.x & 31;
     const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    grid_launch_dependents();
+    grid_dependency_wait();  // drafts and predictions come from the kernels before this one
     if (s >= S) return;
     const int32_t* ds = drafts + (size_t)s * B * w;
     const int32_t* ps = argmax + (size_t)s * B * (w + 1);
@@ -54,10 +56,10 @@ int launch_accept(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_ndraf
                   int B, int w, int32_t* d_hist, int32_t* d_len, int cap, int32_t* d_acc_len, int32_t* d_best_row,
                   int32_t* d_committed, cudaStream_t st) {
     const int warps = 4;
-    accept_commit_kernel<<<(S + warps - 1) / warps, warps * 32, 0, st>>>(
-        d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row, d_committed, ctx->d_status);
+    cudaError_t e = launch_pdl(accept_commit_kernel, dim3((S + warps - 1) / warps), dim3(warps * 32), 0, st, d_drafts, d_ndrafts,
+                               d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row, d_committed, ctx->d_status);
     ctx->launches += 1;
-    return check_cuda(ctx, cudaGetLastError(), "accept_and_commit launch");
+    return check_cuda(ctx, e, "accept_and_commit launch");
 }
 
 }  // namespace ngs

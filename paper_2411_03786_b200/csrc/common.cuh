@@ -5,6 +5,8 @@
 #include <stdint.h>
 #include <stdio.h>
 
+#include <utility>
+
 #include "../../include/ngram_spec.h"
 
 namespace ngs {
@@ -52,6 +54,33 @@ struct spec_ctx {
 };
 
 namespace ngs {
+
+// Launch with programmatic dependent launch allowed: the grid may be scheduled while the previous
+// kernel of the stream is still running (once that kernel has let its dependents go, or has
+// finished), and must execute griddepcontrol.wait before it touches memory the previous work
+// produces.  Behaves like a plain launch after work that never lets dependents go early.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+#ifdef __CUDACC__
+// Wait until the kernels this grid depends on have completed and their writes are visible.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Allow the next kernel in the stream to be scheduled (it still waits before consuming our results).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
 
 int fail(spec_ctx* ctx, int code, const char* fmt, ...);
 int check_cuda(spec_ctx* ctx, cudaError_t e, const char* what);

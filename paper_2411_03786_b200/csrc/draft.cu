@@ -129,6 +129,8 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     const int32_t* __restrict__ h = P.hist + (size_t)s * P.cap;
     const int w = P.w;
 
+    grid_launch_dependents();  // the verify kernel may start streaming weights while this one runs
+    grid_dependency_wait();    // history and lengths come from the previous step's commit
     int L = P.len[s];
     if (L < 0 || L > P.cap) {
         if (tid == 0) atomicOr(P.status, SPEC_STATUS_CAPACITY);
@@ -192,22 +194,31 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                 sm->overflow = 0;
             }
             __syncthreads();
-            // scan: 128-bit loads, four token positions per thread per step, two steps in flight
+            // scan: 128-bit loads, four per thread in flight; positions holding the last token are
+            // collected in a bit mask and handled one by one (they are rare)
             const int4* h4 = reinterpret_cast<const int4*>(h);
             const int n_vec = (n_scan + 3) >> 2;
-            for (int v0 = tid; v0 < n_vec; v0 += 2 * nthr) {
-                int4 va = h4[v0];
-                const int v1 = v0 + nthr;
-                int4 vb = (v1 < n_vec) ? h4[v1] : make_int4(-3, -3, -3, -3);
+            for (int v0 = tid; v0 < n_vec; v0 += 4 * nthr) {
+                int4 vv[4];
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int4 vv = half ? vb : va;
-                    const int xb = (half ? v1 : v0) << 2;
-                    const int toks[4] = {vv.x, vv.y, vv.z, vv.w};
+                for (int u = 0; u < 4; ++u) {
+                    const int vi = v0 + u * nthr;
+                    vv[u] = (vi < n_vec) ? h4[vi] : make_int4(-3, -3, -3, -3);
+                }
+                unsigned hits = 0;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int x = xb + e;
-                        if (toks[e] != t0 || x >= n_scan) continue;
+                for (int u = 0; u < 4; ++u) {
+                    const int xb = (v0 + u * nthr) << 2;
+                    hits |= (unsigned)(vv[u].x == t0 && xb + 0 < n_scan) << (4 * u + 0);
+                    hits |= (unsigned)(vv[u].y == t0 && xb + 1 < n_scan) << (4 * u + 1);
+                    hits |= (unsigned)(vv[u].z == t0 && xb + 2 < n_scan) << (4 * u + 2);
+                    hits |= (unsigned)(vv[u].w == t0 && xb + 3 < n_scan) << (4 * u + 3);
+                }
+                while (hits) {
+                    const int bit = __ffs(hits) - 1;
+                    hits &= hits - 1;
+                    {
+                        const int x = ((v0 + (bit >> 2) * nthr) << 2) + (bit & 3);
                         // length of the common suffix of hist[0..x] and the whole history, up to q_max
                         int m = 1;
                         if (P.q_max > 1 && x >= 1 && h[x - 1] == t1) {
@@ -437,9 +448,9 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
         if (rc) return rc;
         attr_done = true;
     }
-    draft_kernel<<<S, threads, smem, st>>>(P);
+    cudaError_t e = launch_pdl(draft_kernel, dim3(S), dim3(threads), smem, st, P);
     ctx->launches += 1;
-    return check_cuda(ctx, cudaGetLastError(), "draft_context_ngrams launch");
+    return check_cuda(ctx, e, "draft_context_ngrams launch");
 }
 
 }  // namespace ngs

@@ -214,6 +214,37 @@ struct UnitIter {
     }
 };
 
+// The producer's view of the same order, one k-block at a time.
+struct KbCursor {
+    UnitIter it;
+    Unit un;
+    int b0, nb, kb;
+    bool valid;
+    __device__ __forceinline__ KbCursor(const GemmParams& p, int max_boxes) : it(p), b0(0), nb(0), kb(0), valid(false) {
+        next_unit(p, max_boxes);
+    }
+    __device__ __forceinline__ void next_unit(const GemmParams& p, int max_boxes) {
+        do {
+            valid = it.next(p, un);
+        } while (valid && un.box_begin >= un.box_end);
+        if (valid) {
+            b0 = un.box_begin;
+            nb = min(max_boxes, un.box_end - b0);
+            kb = 0;
+        }
+    }
+    __device__ __forceinline__ void advance(const GemmParams& p, int max_boxes) {
+        if (++kb < p.num_kb) return;
+        kb = 0;
+        b0 += max_boxes;
+        if (b0 < un.box_end) {
+            nb = min(max_boxes, un.box_end - b0);
+            return;
+        }
+        next_unit(p, max_boxes);
+    }
+};
+
 // ------------------------------------------------------------------------------------------ the kernel
 // KT = capacity of the per-thread top-k list (registers); only MODE_TOPK uses it.
 template <int MODE, int KT>
@@ -260,6 +291,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) grid_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -268,29 +300,35 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
-            UnitIter it(p);
-            Unit un;
             const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2;
-            while (ok && it.next(p, un)) {
-                for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES) {
-                    const int nb = min(MAX_BOXES, un.box_end - b0);
-                    for (int kb = 0; kb < p.num_kb; ++kb) {
-                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) {
-                            ok = false;
-                            break;
-                        }
-                        const uint32_t full = bar_full + 8 * stage;
-                        const uint32_t sa = tiles + stage * STAGE_BYTES;
-                        mbar_expect_tx(full, a_box_bytes + (uint32_t)(nb * BOX_BYTES));
-                        tma_load_2d(sa, &tmA, kb * BLOCK_K, un.m_tile * BLOCK_M, full);
-                        for (int j = 0; j < nb; ++j)
-                            tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, kb * BLOCK_K, (b0 + j) * BOX_N, full);
-                        ++issued;
-                        if (++stage == STAGES) {
-                            stage = 0;
-                            phase ^= 1u;
-                        }
+            // W is a constant of the model: fill the ring with its tiles before waiting for the kernel
+            // that produces the activations, then add the A tiles of those stages.
+            int n_pref = 0;
+            for (KbCursor pre(p, MAX_BOXES); n_pref < STAGES && pre.valid; pre.advance(p, MAX_BOXES), ++n_pref) {
+                const uint32_t full = bar_full + 8 * n_pref;
+                const uint32_t sa = tiles + n_pref * STAGE_BYTES;
+                mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_BYTES));
+                for (int j = 0; j < pre.nb; ++j)
+                    tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, pre.kb * BLOCK_K, (pre.b0 + j) * BOX_N, full);
+            }
+            grid_dependency_wait();
+            for (KbCursor cur(p, MAX_BOXES); cur.valid; cur.advance(p, MAX_BOXES)) {
+                const uint32_t full = bar_full + 8 * stage;
+                const uint32_t sa = tiles + stage * STAGE_BYTES;
+                if (issued >= n_pref) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
                     }
+                    mbar_expect_tx(full, a_box_bytes + (uint32_t)(cur.nb * BOX_BYTES));
+                    for (int j = 0; j < cur.nb; ++j)
+                        tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + j) * BOX_N, full);
+                }
+                tma_load_2d(sa, &tmA, cur.kb * BLOCK_K, cur.un.m_tile * BLOCK_M, full);
+                ++issued;
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1u;
                 }
             }
             if (!ok) {
@@ -357,6 +395,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
         uint32_t tile = 0;
         bool ok = true;
+        grid_dependency_wait();  // the outputs and the merge scratch may still be in use by the previous kernel
         UnitIter it(p);
         Unit un;
         while (ok && it.next(p, un)) {
@@ -684,9 +723,9 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     fill_common(ctx, p, M, sh);
     p.argmax = d_argmax;
     p.maxv = d_max;
-    head_gemm_kernel<MODE_ARGMAX, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
+    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, tmA, *tmW, p);
     ctx->launches += 1;
-    return check_cuda(ctx, cudaGetLastError(), "verify_lmhead_argmax launch");
+    return check_cuda(ctx, e, "verify_lmhead_argmax launch");
 }
 
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st) {
