@@ -77,6 +77,7 @@ struct DraftSmem {
 __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int p, int qi, int w, uint32_t hsh,
                                              int slots, int max_groups, int* rep, int* cnt, int* last,
                                              int* grp_slot, DraftSmem* sm) {
+    if (*((volatile int*)&sm->overflow)) return;  // this pass is void already: do not fill the table further
     uint32_t slot = hsh & (uint32_t)(slots - 1);
     const int me = (qi << 28) | p;
     for (int probe = 0; probe < slots; ++probe) {
@@ -199,6 +200,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             const int4* h4 = reinterpret_cast<const int4*>(h);
             const int n_vec = (n_scan + 3) >> 2;
             for (int v0 = tid; v0 < n_vec; v0 += 4 * nthr) {
+                if (*((volatile int*)&sm->overflow)) break;  // too many groups for one pass: rescan with more passes
                 int4 vv[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -432,8 +434,8 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.src = d_src;
     P.counts = d_counts;
     P.status = ctx->d_status;
-    int slots = 1024;
-    while (slots < cap && slots < 8192) slots <<= 1;
+    int slots = 1024;  // at most slots / 2 distinct continuations are grouped in one pass
+    while (slots < cap / 2 && slots < 8192) slots <<= 1;
     P.slots = slots;
     P.max_groups = slots / 2;
     const int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);
