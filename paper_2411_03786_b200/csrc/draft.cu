@@ -62,8 +62,10 @@ struct DraftSmem {
     int32_t cand_cnt[kMaxCand];
     int32_t cand_keep[kMaxCand];
     int32_t row_of[kMaxB];                      // candidate that became draft row b
+    int32_t row_of_tmp[kMaxCand];               // duplicate flags
     int cand_off[kMaxNQ + 2];
     int n_cnt[kMaxNQ];
+    int rank_acc[kRankMax];   // groups of the same query length with a larger key
     int32_t chain[kMaxKTab][kMaxW];
     int chain_ok[kMaxKTab];
     int n_run[kMaxNQ];
@@ -151,11 +153,15 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             bool ok = true;
             if (P.ext != nullptr && w <= P.w_ext) {
                 const int32_t* e = P.ext + ((size_t)x * P.k_tab + lane) * P.w_ext;
-                for (int j = 0; j < w; ++j) {
-                    int t = e[j];
-                    ok = ok && (t >= 0 && t < P.V);
-                    sm->chain[lane][j] = t;
-                }
+                int t[kMaxW];  // all loads first, so they are in flight together
+#pragma unroll
+                for (int j = 0; j < kMaxW; ++j) t[j] = (j < w) ? e[j] : 0;
+#pragma unroll
+                for (int j = 0; j < kMaxW; ++j)
+                    if (j < w) {
+                        ok = ok && (t[j] >= 0 && t[j] < P.V);
+                        sm->chain[lane][j] = t[j];
+                    }
             } else {
                 int t = P.tab[(size_t)x * P.k_tab + lane];
                 for (int j = 0; j < w; ++j) {
@@ -249,29 +255,44 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                 break;
             }
             if (R == 1 && sm->n_groups <= kRankMax) {
-                // Few groups (the usual case): every thread ranks groups by counting the groups of the same
-                // query length with a larger (count, start) key; rank r < topk lands in slot r.
+                // Few groups (the usual case).
+                // Every group is ranked by counting the groups of the same query length with a larger
+                // (count, start) key; the comparisons of one group are split over `parts` threads so that
+                // all threads stay busy.  Rank r < topk lands in slot r.
                 const int n_groups = sm->n_groups;
                 if (tid < kMaxNQ) sm->n_cnt[tid] = 0;
                 for (int g = tid; g < n_groups; g += nthr) {
                     const int slot = grp_slot[g];
                     const unsigned long long qi = (unsigned long long)(rep[slot] >> 28);
                     sm->gkey[g] = (qi << 60) | ((unsigned long long)(uint32_t)cnt[slot] << 32) | (uint32_t)last[slot];
+                    sm->rank_acc[g] = 0;
+                }
+                __syncthreads();
+                int parts = 1;
+                while (parts < 8 && n_groups * parts < 2 * nthr) parts <<= 1;
+                const int span = (n_groups + parts - 1) / parts;
+                for (int item = tid; item < n_groups * parts; item += nthr) {
+                    const int g = item / parts, part = item - g * parts;
+                    const unsigned long long mine = sm->gkey[g];
+                    const int o_end = min(n_groups, (part + 1) * span);
+                    int rank = 0;
+                    for (int o = part * span; o < o_end; ++o) {
+                        const unsigned long long other = sm->gkey[o];
+                        rank += ((other >> 60) == (mine >> 60) && other > mine) ? 1 : 0;
+                    }
+                    if (rank) atomicAdd(&sm->rank_acc[g], rank);
                 }
                 __syncthreads();
                 for (int g = tid; g < n_groups; g += nthr) {
                     const unsigned long long mine = sm->gkey[g];
-                    int rank = 0;
-                    for (int o = 0; o < n_groups; ++o) {
-                        const unsigned long long other = sm->gkey[o];
-                        rank += ((other >> 60) == (mine >> 60) && other > mine) ? 1 : 0;
+                    const int rank = sm->rank_acc[g];
+                    if (rank < P.topk) {  // ranks are distinct, so the rows kept are 0 .. max rank
+                        sm->run_key[(int)(mine >> 60)][rank] = mine & 0x0FFFFFFFFFFFFFFFull;
+                        atomicMax(&sm->n_cnt[(int)(mine >> 60)], rank + 1);
                     }
-                    const int qi = (int)(mine >> 60);
-                    atomicAdd(&sm->n_cnt[qi], 1);
-                    if (rank < P.topk) sm->run_key[qi][rank] = mine & 0x0FFFFFFFFFFFFFFFull;
                 }
                 __syncthreads();
-                if (tid < kMaxNQ) sm->n_run[tid] = min(P.topk, sm->n_cnt[tid]);
+                if (tid < kMaxNQ) sm->n_run[tid] = sm->n_cnt[tid];
             } else if (warp < P.n_q) {
                 // rank this pass's groups together with the winners of earlier passes: warp qi
                 const int qi = warp;
@@ -362,23 +383,25 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     }
     __syncthreads();
     if (dedup) {
-        int drop[(kMaxCand + 127) / 128];  // decisions first, writes after: cand_keep is read by others (>= 128 threads)
-        int n_mine = 0;
-        for (int ci = tid; ci < n_cand; ci += nthr, ++n_mine) {
-            bool dup = false;
-            if (sm->cand_keep[ci])
-                for (int j = 0; j < ci && !dup; ++j) {
-                    if (!sm->cand_keep[j]) continue;  // an invalid model row
-                    bool same = true;
-                    for (int t = 0; t < w && same; ++t) same = cand[j * w + t] == cand[ci * w + t];
-                    dup = same;
-                }
-            drop[n_mine] = dup ? 1 : 0;
+        // all (earlier, later) pairs side by side; a later row equal to an earlier valid row is dropped
+        int32_t* dropped = sm->row_of_tmp;
+        for (int i = tid; i < n_cand; i += nthr) dropped[i] = 0;
+        __syncthreads();
+        const int n_pairs = n_cand * (n_cand - 1) / 2;
+        for (int pi = tid; pi < n_pairs; pi += nthr) {
+            // pair index -> (ci, j) with j < ci: ci is the largest integer with ci (ci - 1) / 2 <= pi
+            int ci = (int)((1.0f + sqrtf(1.0f + 8.0f * (float)pi)) * 0.5f);
+            while (ci * (ci - 1) / 2 > pi) --ci;
+            while ((ci + 1) * ci / 2 <= pi) ++ci;
+            const int j = pi - ci * (ci - 1) / 2;
+            if (!sm->cand_keep[ci] || !sm->cand_keep[j]) continue;
+            bool same = true;
+            for (int t = 0; t < w && same; ++t) same = cand[j * w + t] == cand[ci * w + t];
+            if (same) dropped[ci] = 1;
         }
         __syncthreads();
-        n_mine = 0;
-        for (int ci = tid; ci < n_cand; ci += nthr, ++n_mine)
-            if (drop[n_mine]) sm->cand_keep[ci] = 0;
+        for (int i = tid; i < n_cand; i += nthr)
+            if (dropped[i]) sm->cand_keep[i] = 0;
         __syncthreads();
     }
     if (warp == 0) {
