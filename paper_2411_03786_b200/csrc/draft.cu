@@ -1,4 +1,6 @@
-// Context N-gram drafting and mixed allocation: one CTA per sequence.
+// Context N-gram drafting and mixed allocation: one CTA per sequence, or for long histories one
+// thread-block cluster per sequence whose CTAs each scan a slice of the history and group their
+// matches in the leader CTA's hash table through distributed shared memory.
 //
 // One streaming pass over the history serves every query length at once.  A position p is the
 // start of a continuation for query length q when the q tokens before p equal the last q tokens
@@ -8,7 +10,11 @@
 // actual tokens, so grouping is exact.  If a sequence has more distinct continuations than the
 // table holds, the scan is repeated in R passes, pass r keeping only the groups whose hash falls
 // in residue class r, and the per-pass winners are merged: still exact, only slower.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace ngs {
 
@@ -126,9 +132,21 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     int* last = cnt + P.slots;
     int* grp_slot = last + P.slots;
 
+    // The cluster's CTAs share one sequence; rank 0 (the leader) owns the table and writes the result.
+    // Every cluster-wide barrier below is reached by all CTAs: the loop bounds depend only on the
+    // sequence length, the launch parameters and a flag every CTA reads between two barriers.
+    cg::cluster_group cluster = cg::this_cluster();
+    const int csize = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
+    const bool leader = crank == 0;
+    DraftSmem* lsm = cluster.map_shared_rank(sm, 0);
+    int* lrep = cluster.map_shared_rank(rep, 0);
+    int* lcnt = cluster.map_shared_rank(cnt, 0);
+    int* llast = cluster.map_shared_rank(last, 0);
+    int* lgrp_slot = cluster.map_shared_rank(grp_slot, 0);
+
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
-    const int s = blockIdx.x;
+    const int s = (int)blockIdx.x / csize;
     const int32_t* __restrict__ h = P.hist + (size_t)s * P.cap;
     const int w = P.w;
 
@@ -136,7 +154,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     grid_dependency_wait();    // history and lengths come from the previous step's commit
     int L = P.len[s];
     if (L < 0 || L > P.cap) {
-        if (tid == 0) atomicOr(P.status, SPEC_STATUS_CAPACITY);
+        if (tid == 0 && leader) atomicOr(P.status, SPEC_STATUS_CAPACITY);
         L = 0;
     }
     if (tid < kMaxQ) sm->tq[tid] = (tid < L) ? h[L - 1 - tid] : -2;
@@ -145,7 +163,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     __syncthreads();
 
     // ---- extended model bigram of the last token (rank r on lane r), overlapped with the scan
-    if (warp == nwarps - 1 && (P.flags & SPEC_FLAG_MODEL_FILL) && L >= 1) {
+    if (leader && warp == nwarps - 1 && (P.flags & SPEC_FLAG_MODEL_FILL) && L >= 1) {
         const int x = sm->tq[0];
         if (x < 0 || x >= P.V) {
             if (lane == 0) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
@@ -191,22 +209,26 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         if (tid < kMaxNQ) sm->n_run[tid] = 0;
         bool overflowed = false;
         for (int r = 0; r < R && !overflowed; ++r) {
-            for (int i = tid; i < P.slots; i += nthr) {
-                rep[i] = -1;
-                cnt[i] = 0;
-                last[i] = -1;
+            if (leader) {
+                for (int i = tid; i < P.slots; i += nthr) {
+                    rep[i] = -1;
+                    cnt[i] = 0;
+                    last[i] = -1;
+                }
+                if (tid == 0) {
+                    sm->n_groups = 0;
+                    sm->overflow = 0;
+                }
             }
-            if (tid == 0) {
-                sm->n_groups = 0;
-                sm->overflow = 0;
-            }
-            __syncthreads();
+            cluster.sync();  // the leader's table is ready
             // scan: 128-bit loads, four per thread in flight; positions holding the last token are
             // collected in a bit mask and handled one by one (they are rare)
             const int4* h4 = reinterpret_cast<const int4*>(h);
-            const int n_vec = (n_scan + 3) >> 2;
-            for (int v0 = tid; v0 < n_vec; v0 += 4 * nthr) {
-                if (*((volatile int*)&sm->overflow)) break;  // too many groups for one pass: rescan with more passes
+            const int n_vec_all = (n_scan + 3) >> 2;
+            const int v_chunk = (n_vec_all + csize - 1) / csize;  // this CTA's slice of the history
+            const int n_vec = min(n_vec_all, (crank + 1) * v_chunk);
+            for (int v0 = crank * v_chunk + tid; v0 < n_vec; v0 += 4 * nthr) {
+                if (*((volatile int*)&lsm->overflow)) break;  // too many groups for one pass: rescan with more passes
                 int4 vv[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -244,16 +266,19 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                             if (m < q || L < q + w) continue;
                             const uint32_t hq = fmix32(hc + (uint32_t)qi * 0x632BE5ABu);
                             if (R > 1 && (int)(fmix32(hq ^ 0xA511E9B3u) % (uint32_t)R) != r) continue;
-                            insert_match(h, p, qi, w, hq, P.slots, P.max_groups, rep, cnt, last, grp_slot, sm);
+                            insert_match(h, p, qi, w, hq, P.slots, P.max_groups, lrep, lcnt, llast, lgrp_slot, lsm);
                         }
                     }
                 }
             }
-            __syncthreads();
-            if (sm->overflow) {
+            cluster.sync();  // every CTA's matches are in the table
+            const int ov = *((volatile int*)&lsm->overflow);
+            cluster.sync();  // every CTA has read the flag before the leader may reset it
+            if (ov) {
                 overflowed = true;
                 break;
             }
+            if (!leader) continue;
             if (R == 1 && sm->n_groups <= kRankMax) {
                 // Few groups (the usual case).
                 // Every group is ranked by counting the groups of the same query length with a larger
@@ -334,6 +359,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             break;
         }
     }
+    if (!leader) return;  // nobody reads a non-leader's shared memory, and no cluster barrier follows
     __syncthreads();
     if (gave_up) {
         if (tid < kMaxNQ) sm->n_run[tid] = 0;
@@ -462,6 +488,8 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.slots = slots;
     P.max_groups = slots / 2;
     const int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);
+    unsigned csize = 1;  // CTAs per sequence: one per 16K tokens of capacity, at most 8
+    while (csize < 8 && (int)(csize * 2) * 16384 <= cap) csize <<= 1;
     const size_t table_bytes = (size_t)slots * 3 * sizeof(int) + (size_t)P.max_groups * sizeof(int);
     const size_t cand_bytes = (size_t)(n_q * topk + kMaxKTab) * w * sizeof(int32_t);  // aliases the table
     const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + (table_bytes > cand_bytes ? table_bytes : cand_bytes);
@@ -473,7 +501,7 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
         if (rc) return rc;
         attr_done = true;
     }
-    cudaError_t e = launch_pdl(draft_kernel, dim3(S), dim3(threads), smem, st, P);
+    cudaError_t e = launch_pdl_cluster(draft_kernel, dim3((unsigned)S * csize), dim3(threads), smem, st, csize, P);
     ctx->launches += 1;
     return check_cuda(ctx, e, "draft_context_ngrams launch");
 }
