@@ -488,8 +488,10 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.slots = slots;
     P.max_groups = slots / 2;
     const int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);
-    unsigned csize = 1;  // CTAs per sequence: one per 16K tokens of capacity, at most 8
-    while (csize < 8 && (int)(csize * 2) * 16384 <= cap) csize <<= 1;
+    // CTAs per sequence: one per 16K tokens of capacity, at most 8, and only while the batch alone
+    // cannot fill the GPU (with many sequences one CTA each is the faster way to stream them)
+    unsigned csize = 1;
+    while (csize < 8 && (int)(csize * 2) * 16384 <= cap && (long long)S * (csize * 2) <= ctx->num_sms) csize <<= 1;
     const size_t table_bytes = (size_t)slots * 3 * sizeof(int) + (size_t)P.max_groups * sizeof(int);
     const size_t cand_bytes = (size_t)(n_q * topk + kMaxKTab) * w * sizeof(int32_t);  // aliases the table
     const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + (table_bytes > cand_bytes ? table_bytes : cand_bytes);
