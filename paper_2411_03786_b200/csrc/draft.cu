@@ -23,7 +23,7 @@ struct DraftParams {
     const int32_t* len;
     int S, cap;
     int qs[kMaxNQ];
-    int n_q, q_max;
+    int n_q, q_max, q_min;
     int topk, B, w, flags;
     const int32_t* tab;
     int k_tab;
@@ -227,8 +227,11 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             const int n_vec_all = (n_scan + 3) >> 2;
             const int v_chunk = (n_vec_all + csize - 1) / csize;  // this CTA's slice of the history
             const int n_vec = min(n_vec_all, (crank + 1) * v_chunk);
-            for (int v0 = crank * v_chunk + tid; v0 < n_vec; v0 += 4 * nthr) {
-                if (*((volatile int*)&lsm->overflow)) break;  // too many groups for one pass: rescan with more passes
+            const bool need2 = P.q_min >= 2;  // every query has at least two tokens: test the second one in registers
+            for (int vw = crank * v_chunk + (tid - lane); vw < n_vec; vw += 4 * nthr) {  // warp-uniform trip count
+                // too many groups for one pass: rescan with more passes
+                if (__any_sync(0xffffffffu, *((volatile int*)&lsm->overflow))) break;
+                const int v0 = vw + lane;
                 int4 vv[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -238,11 +241,21 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                 unsigned hits = 0;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int xb = (v0 + u * nthr) << 2;
-                    hits |= (unsigned)(vv[u].x == t0 && xb + 0 < n_scan) << (4 * u + 0);
-                    hits |= (unsigned)(vv[u].y == t0 && xb + 1 < n_scan) << (4 * u + 1);
-                    hits |= (unsigned)(vv[u].z == t0 && xb + 2 < n_scan) << (4 * u + 2);
-                    hits |= (unsigned)(vv[u].w == t0 && xb + 3 < n_scan) << (4 * u + 3);
+                    const int vi = v0 + u * nthr;
+                    const int xb = vi << 2;
+                    bool px = true, py = true, pz = true, pw = true;
+                    if (need2) {  // token before each position: from this vector, or from the lane to the left
+                        int before = __shfl_up_sync(0xffffffffu, vv[u].w, 1);
+                        if (lane == 0) before = (vi > 0 && vi < n_vec) ? h[xb - 1] : -5;
+                        px = before == t1;
+                        py = vv[u].x == t1;
+                        pz = vv[u].y == t1;
+                        pw = vv[u].z == t1;
+                    }
+                    hits |= (unsigned)(vv[u].x == t0 && px && xb + 0 < n_scan) << (4 * u + 0);
+                    hits |= (unsigned)(vv[u].y == t0 && py && xb + 1 < n_scan) << (4 * u + 1);
+                    hits |= (unsigned)(vv[u].z == t0 && pz && xb + 2 < n_scan) << (4 * u + 2);
+                    hits |= (unsigned)(vv[u].w == t0 && pw && xb + 3 < n_scan) << (4 * u + 3);
                 }
                 while (hits) {
                     const int bit = __ffs(hits) - 1;
@@ -465,9 +478,11 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.cap = cap;
     P.n_q = n_q;
     P.q_max = 0;
+    P.q_min = kMaxQ;
     for (int i = 0; i < kMaxNQ; ++i) {
         P.qs[i] = i < n_q ? qs[i] : 0;
         if (i < n_q && qs[i] > P.q_max) P.q_max = qs[i];
+        if (i < n_q && qs[i] < P.q_min) P.q_min = qs[i];
     }
     P.topk = topk;
     P.B = B;
