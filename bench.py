@@ -472,7 +472,7 @@ def main():
 
 # DRAM bytes per verify launch from the ncu captures summarised under profiles/ (None = not captured
 # for the current kernel).
-TRAFFIC = {}
+TRAFFIC = {"C2": 266.7e6, "C3": 1.655e9}
 
 
 def run_reference(args, c, cfg):
