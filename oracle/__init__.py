@@ -152,6 +152,25 @@ def verify(H, W, rows=None):
     return am, mx, gap
 
 
+def unigram_dist2(W, E, rows=None) -> np.ndarray:
+    """Section 4.1 "Unigram": squared distance of each output embedding from the mean, in the metric
+    induced by the input embeddings (centred rows rounded to bf16, the rest fp64)."""
+    W, E = _u16(W), _u16(E)
+    V, d = W.shape
+    r, n = _rowsel(rows, V)
+    out = np.empty(n, dtype=np.float64)
+    lib().oracle_unigram_dist2(_p(W, C.c_uint16), _p(E, C.c_uint16), V, d, _p(r, C.c_int64), n, _p(out, C.c_double))
+    return out
+
+
+def smallest_k(dist2, k: int) -> np.ndarray:
+    """Top-k unigram tokens: smallest distance first, equal distances by ascending id."""
+    dist2 = np.ascontiguousarray(dist2, dtype=np.float64)
+    idx = np.empty(k, dtype=np.int32)
+    lib().oracle_smallest_k(_p(dist2, C.c_double), int(dist2.size), int(k), _p(idx, C.c_int32))
+    return idx
+
+
 def accept_commit(drafts, n_drafts, P, hist, lens):
     """Greedy acceptance + commit.  ``hist`` and ``lens`` are updated in place.
 

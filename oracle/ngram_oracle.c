@@ -268,6 +268,52 @@ void oracle_verify_rows(const uint16_t* H, const int64_t* rowsel, int n_rows, co
     }
 }
 
+/* ------------------------------------------------------------------ model unigram (Section 4.1, "Unigram")
+ *
+ * d(x) = || u_x - ubar ||_V where u_x is row x of the output embedding W, ubar the mean row, and the
+ * norm comes from <a, b>_V = sum_y (a . v_y)(b . v_y) over the rows v_y of the input embedding E.
+ * So d(x)^2 = sum_y ((u_x - ubar) . v_y)^2; p(x) is proportional to exp(-d(x)): the top-k unigram
+ * tokens are those with the smallest d (equal values by ascending token id).
+ * The centred rows are rounded once to bfloat16 (they feed a bf16 tensor-core contraction), everything
+ * else is fp64.  rowsel (or NULL) picks the rows x that are evaluated; dist2 is [n_rows].
+ */
+void oracle_unigram_dist2(const uint16_t* W, const uint16_t* E, int V, int d, const int64_t* rowsel, int n_rows,
+                          double* dist2) {
+    double* mean = (double*)calloc((size_t)d, sizeof(double));
+    for (int x = 0; x < V; ++x)
+        for (int t = 0; t < d; ++t) mean[t] += bf16_to_double(W[(long)x * d + t]);
+    for (int t = 0; t < d; ++t) mean[t] /= (double)V;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        long x = rowsel ? (long)rowsel[r] : r;
+        double* c = (double*)malloc(sizeof(double) * (size_t)d);
+        for (int t = 0; t < d; ++t)
+            c[t] = bf16_to_double(oracle_f32_to_bf16((float)(bf16_to_double(W[x * d + t]) - mean[t])));
+        double acc = 0.0;
+        for (int y = 0; y < V; ++y) {
+            double dot = 0.0;
+            for (int t = 0; t < d; ++t) dot += c[t] * bf16_to_double(E[(long)y * d + t]);
+            acc += dot * dot;
+        }
+        dist2[r] = acc;
+        free(c);
+    }
+    free(mean);
+}
+
+/* The k tokens with the smallest distance, ascending; equal distances by ascending token id. */
+void oracle_smallest_k(const double* dist2, int V, int k, int32_t* idx) {
+    char* used = (char*)calloc((size_t)V, 1);
+    for (int j = 0; j < k; ++j) {
+        int best = -1;
+        for (int x = 0; x < V; ++x)
+            if (!used[x] && (best < 0 || dist2[x] < dist2[best])) best = x;
+        idx[j] = best;
+        if (best >= 0) used[best] = 1;
+    }
+    free(used);
+}
+
 /* ------------------------------------------------------------------ greedy acceptance (Sections 1, 5 and Appendix D)
  *
  * Row b of the verify block is [x_L, s_1 .. s_w]; P[b][j] is the model's greedy
