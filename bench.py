@@ -277,7 +277,14 @@ def main():
             ts.append(a.elapsed_time(b))
         ms = min(ts)
         fl = 2.0 * c["V"] * c["V"] * c["d"]
-        table = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_burst_peak": fl / ms / 1e9 / pk["tc_burst"],
+        a, b = ev(), ev()
+        ctx.build_model_unigram(25)
+        a.record()
+        ctx.build_model_unigram(25)
+        b.record()
+        torch.cuda.synchronize()
+        uni_ms = a.elapsed_time(b)
+        table = {"ms": ms, "tflops": fl / ms / 1e9, "unigram_ms": uni_ms, "unigram_tflops": fl / uni_ms / 1e9, "frac_of_burst_peak": fl / ms / 1e9 / pk["tc_burst"],
                  "frac_of_sustained_peak": fl / ms / 1e9 / pk["tc_sustained"], "flops": fl, "peak_source": pk["source"]}
 
     # ---- inputs of a step: histories, then hidden states planted on the initial drafts

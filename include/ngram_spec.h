@@ -98,6 +98,18 @@ const char* spec_last_error(spec_ctx* ctx);
 int build_model_ngram_tables(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx,
                              float* d_tab_val, int32_t* d_ext, void* stream);
 
+/*
+ * Model unigram (Section 4.1 "Unigram").  d(x) = || u_x - ubar ||_V: u_x is row x of the unembedding,
+ * ubar the mean row, and the norm is induced by <a, b>_V = sum_y (a . v_y)(b . v_y) over the rows v_y
+ * of the embedding.  p(x) is proportional to exp(-d(x)), so the top-k unigram tokens are the k with the
+ * smallest d.  The centred rows are rounded once to bfloat16 and contracted with the embedding on the
+ * tensor cores (fp32 accumulation); the [V, V] products are squared and summed in the epilogue.
+ *   d_dist2    [V] float32 out: d(x)^2.
+ *   d_uni_idx  [k_uni] int32 out: tokens by ascending d, equal values by ascending id (k_uni = 0: skip).
+ * Allocates (and keeps) a [V, d] bfloat16 scratch for the centred rows on first use.
+ */
+int build_model_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2, void* stream);
+
 /* Adopt a table built earlier (e.g. loaded from disk) instead of building it. */
 int spec_set_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, const int32_t* d_ext, int w_ext);
 

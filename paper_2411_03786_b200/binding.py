@@ -44,6 +44,7 @@ def load_library(build: bool = True) -> C.CDLL:
     lib.spec_last_error.argtypes = [vp]
     lib.spec_last_error.restype = C.c_char_p
     lib.build_model_ngram_tables.argtypes = [vp, vp, C.c_int, C.c_int, i32p, fp, i32p, vp]
+    lib.build_model_unigram.argtypes = [vp, C.c_int, i32p, fp, vp]
     lib.spec_set_model_table.argtypes = [vp, i32p, C.c_int, i32p, C.c_int]
     lib.draft_context_ngrams.argtypes = [vp, i32p, i32p, C.c_int, C.c_int, ip, C.c_int, C.c_int, C.c_int, C.c_int,
                                          C.c_int, i32p, i32p, i32p, i32p, vp]
@@ -122,6 +123,14 @@ class SpecContext:
                                                        _ptr(val), _ptr(ext), _stream()), "build_model_ngram_tables")
         self._keep_table = (tab, ext, rows)
         return tab, val, ext
+
+    def build_model_unigram(self, k_uni: int):
+        """Returns ``(ids[k_uni] by ascending distance, dist2[V])``."""
+        dev = self._keep[0].device
+        idx = torch.empty(max(k_uni, 1), dtype=torch.int32, device=dev)
+        dist2 = torch.empty(self.V, dtype=torch.float32, device=dev)
+        self._check(self._lib.build_model_unigram(self._h, k_uni, _ptr(idx), _ptr(dist2), _stream()), "build_model_unigram")
+        return idx[:k_uni], dist2
 
     def set_model_table(self, tab: torch.Tensor, ext: torch.Tensor | None = None):
         k_tab = int(tab.shape[1])

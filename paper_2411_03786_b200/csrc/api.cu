@@ -137,6 +137,8 @@ int spec_destroy(spec_ctx* ctx) {
     cudaFree(ctx->d_status);
     cudaFree(ctx->d_keys);
     cudaFree(ctx->d_ticket);
+    cudaFree(ctx->d_centred);
+    cudaFree(ctx->d_colsum);
     cudaFree(ctx->d_part_val);
     cudaFree(ctx->d_part_idx);
     delete ctx;
@@ -225,6 +227,15 @@ int accept_and_commit(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_n
     cudaSetDevice(ctx->device);
     return launch_accept(ctx, d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row,
                          d_committed, (cudaStream_t)stream);
+}
+
+int build_model_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "build_model_unigram: ctx is NULL");
+    if (!d_dist2) return fail(ctx, SPEC_ERR_ARG, "build_model_unigram: d_dist2 is NULL");
+    if (k_uni < 0 || k_uni > 1024 || k_uni > ctx->V || (k_uni > 0 && !d_uni_idx))
+        return fail(ctx, SPEC_ERR_ARG, "build_model_unigram: need 0 <= k_uni <= min(1024, V) and d_uni_idx for k_uni > 0");
+    cudaSetDevice(ctx->device);
+    return launch_unigram(ctx, k_uni, d_uni_idx, d_dist2, (cudaStream_t)stream);
 }
 
 int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, void* stream) {

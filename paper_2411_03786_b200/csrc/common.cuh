@@ -49,6 +49,10 @@ struct spec_ctx {
     // encoded on first use (host-side work only)
     CUtensorMap tm_w[5];
     bool tm_w_ready[5] = {false, false, false, false, false};
+    CUtensorMap tm_e[5];  // same for the embedding (B operand of the unigram contraction)
+    bool tm_e_ready[5] = {false, false, false, false, false};
+    void* d_centred = nullptr;  // unigram scratch: bf16 [V, d] output embeddings minus their mean
+    float* d_colsum = nullptr;  // unigram scratch: [64 + 1, d] partial column sums and the mean
     long long launches = 0;
     char err[256] = {0};
 };
@@ -115,6 +119,7 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
 int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
                  int32_t* d_ext, cudaStream_t st);
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st);
+int launch_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2, cudaStream_t st);
 // draft.cu / accept.cu
 int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
                  int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,

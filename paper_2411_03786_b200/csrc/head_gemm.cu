@@ -4,6 +4,7 @@
 //   MODE_ARGMAX  verification: per row of A the arg max over the vocabulary   (verify_lmhead_argmax)
 //   MODE_TOPK    model bigram table: per row the k largest entries           (build_model_ngram_tables)
 //   MODE_STORE   plain fp32 store, for the logits tolerance check            (spec_debug_logits)
+//   MODE_SUMSQ   model unigram: per row the sum of squares over all columns  (build_model_unigram)
 //
 // A is [a_rows, d] and W is [V, d], both bf16 and K-major, so both operands use the same
 // 128-byte-swizzled K-major shared-memory layout.  One CTA owns the accumulator of a
@@ -47,7 +48,7 @@ constexpr int TMEM_COLS = 512;
 constexpr int GEMM_THREADS = 192;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
-enum { MODE_ARGMAX = 0, MODE_TOPK = 1, MODE_STORE = 2 };
+enum { MODE_ARGMAX = 0, MODE_TOPK = 1, MODE_STORE = 2, MODE_SUMSQ = 3 };
 
 struct GemmParams {
     int a_rows;    // rows of A
@@ -401,7 +402,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         while (ok && it.next(p, un)) {
             const int row = un.m_tile * BLOCK_M + row_in_tile;
             // running reduction of this row over the unit's columns
-            float best_v = -INFINITY;
+            float best_v = MODE == MODE_SUMSQ ? 0.0f : -INFINITY;
             int best_i = 0x7FFFFFFF;
             // Sorted list, value descending, statically indexed so it stays in registers.  The k_tab live
             // entries sit at the bottom [KT - k_tab, KT); the slots above hold +inf, which nothing beats,
@@ -464,6 +465,12 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                 }
                             }
                         }
+                    } else if (MODE == MODE_SUMSQ) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float v = __uint_as_float(r[j]);
+                            if (j < lim) best_v += v * v;  // best_v doubles as the running sum (starts at 0)
+                        }
                     } else {
                         if (row < p.a_rows) {
                             float* out = p.logits + (size_t)row * p.V + cbase;
@@ -483,6 +490,8 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const unsigned long long key =
                         ((unsigned long long)orderable_f32(best_v) << 32) | (unsigned long long)(~(uint32_t)best_i);
                     atomicMax(p.keys + row, key);
+                } else if (MODE == MODE_SUMSQ) {
+                    p.part_val[(size_t)un.chunk * p.a_rows + row] = best_v;
                 } else if (MODE == MODE_TOPK) {
                     const size_t base = ((size_t)un.chunk * p.a_rows + row) * p.k_tab;
 #pragma unroll
@@ -663,14 +672,17 @@ static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks) {
     return s;
 }
 
-// Tensor map of the unembedding for the shape's box size (encoded once per context).
-static int w_map(spec_ctx* ctx, const Shape& sh, const CUtensorMap** out) {
-    if (!ctx->tm_w_ready[sh.box_idx]) {
-        int rc = make_tensor_map(ctx, &ctx->tm_w[sh.box_idx], ctx->unembed, ctx->V, ctx->d, sh.box_n);
+// Tensor map of the unembedding (or, for the unigram, the embedding) for the shape's box size,
+// encoded once per context.
+static int w_map(spec_ctx* ctx, const Shape& sh, const CUtensorMap** out, bool embedding = false) {
+    CUtensorMap* maps = embedding ? ctx->tm_e : ctx->tm_w;
+    bool* ready = embedding ? ctx->tm_e_ready : ctx->tm_w_ready;
+    if (!ready[sh.box_idx]) {
+        int rc = make_tensor_map(ctx, &maps[sh.box_idx], embedding ? ctx->embed : ctx->unembed, ctx->V, ctx->d, sh.box_n);
         if (rc) return rc;
-        ctx->tm_w_ready[sh.box_idx] = true;
+        ready[sh.box_idx] = true;
     }
-    *out = &ctx->tm_w[sh.box_idx];
+    *out = &maps[sh.box_idx];
     return SPEC_OK;
 }
 
@@ -792,6 +804,125 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
         if ((rc = check_cuda(ctx, cudaGetLastError(), "table extension launch"))) return rc;
     }
     return SPEC_OK;
+}
+
+// ------------------------------------------------------------------------------------------ model unigram
+// Column sums of W in two deterministic stages: colsum[y][t] over a slab of rows, then the mean.
+__global__ void unigram_colsum_kernel(const __nv_bfloat16* __restrict__ W, int V, int d, float* __restrict__ colsum) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= d) return;
+    const int rows_per = (V + gridDim.y - 1) / gridDim.y;
+    const int x0 = blockIdx.y * rows_per, x1 = min(V, x0 + rows_per);
+    float acc = 0.0f;
+    for (int x = x0; x < x1; ++x) acc += __bfloat162float(W[(size_t)x * d + t]);
+    colsum[(size_t)blockIdx.y * d + t] = acc;
+}
+__global__ void unigram_mean_kernel(const float* __restrict__ colsum, int n_slabs, int V, int d, float* __restrict__ mean) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= d) return;
+    float acc = 0.0f;
+    for (int y = 0; y < n_slabs; ++y) acc += colsum[(size_t)y * d + t];
+    mean[t] = acc / (float)V;
+}
+// centred[x][t] = bf16(W[x][t] - mean[t])
+__global__ void unigram_centre_kernel(const __nv_bfloat16* __restrict__ W, const float* __restrict__ mean, size_t n, int d,
+                                      __nv_bfloat16* __restrict__ out) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (; i < n; i += stride) out[i] = __float2bfloat16_rn(__bfloat162float(W[i]) - mean[i % d]);
+}
+// dist2[x] = sum over chunks of the partial sums, in chunk order
+__global__ void unigram_sum_kernel(const float* __restrict__ part, int n_chunks, int V, float* __restrict__ dist2) {
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= V) return;
+    float acc = 0.0f;
+    for (int c = 0; c < n_chunks; ++c) acc += part[(size_t)c * V + x];
+    dist2[x] = acc;
+}
+// The k smallest distances in ascending order, equal values by ascending token id: one CTA picks, k
+// times, the smallest (value, id) key above the previous pick.
+__global__ void __launch_bounds__(1024) unigram_smallest_k_kernel(const float* __restrict__ dist2, int V, int k,
+                                                                  int32_t* __restrict__ idx) {
+    __shared__ unsigned long long warp_min[32];
+    __shared__ unsigned long long picked;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned long long prev = 0ull;
+    bool first = true;
+    for (int j = 0; j < k; ++j) {
+        unsigned long long best = ~0ull;
+        for (int x = tid; x < V; x += blockDim.x) {
+            const unsigned long long key = ((unsigned long long)orderable_f32(dist2[x]) << 32) | (uint32_t)x;
+            if ((first || key > prev) && key < best) best = key;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+            best = other < best ? other : best;
+        }
+        if (lane == 0) warp_min[warp] = best;
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long b = lane < (int)(blockDim.x >> 5) ? warp_min[lane] : ~0ull;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long other = __shfl_xor_sync(0xffffffffu, b, o);
+                b = other < b ? other : b;
+            }
+            if (lane == 0) {
+                picked = b;
+                idx[j] = (int32_t)(uint32_t)(b & 0xFFFFFFFFull);
+            }
+        }
+        __syncthreads();
+        prev = picked;
+        first = false;
+        __syncthreads();
+    }
+}
+
+int launch_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2, cudaStream_t st) {
+    int rc = set_smem_attr<MODE_SUMSQ, 1>(ctx);
+    if (rc) return rc;
+    const int V = ctx->V, d = ctx->d, n_slabs = 64;
+    const size_t n = (size_t)V * d;
+    if (!ctx->d_centred) {
+        if ((rc = check_cuda(ctx, cudaMalloc(&ctx->d_centred, n * 2), "cudaMalloc(centred embeddings)"))) return rc;
+        if ((rc = check_cuda(ctx, cudaMalloc(&ctx->d_colsum, sizeof(float) * (size_t)(n_slabs + 1) * d), "cudaMalloc(column sums)")))
+            return rc;
+    }
+    const Shape sh = cached_shape(ctx, V, (size_t)1 << 20);
+    const size_t need = (size_t)sh.n_chunks * V;
+    if (need > ctx->part_capacity) {
+        cudaStreamSynchronize(st);
+        cudaFree(ctx->d_part_val);
+        cudaFree(ctx->d_part_idx);
+        ctx->d_part_val = nullptr;
+        ctx->d_part_idx = nullptr;
+        ctx->part_capacity = 0;
+        if ((rc = check_cuda(ctx, cudaMalloc(&ctx->d_part_val, need * sizeof(float)), "cudaMalloc(partial sums)"))) return rc;
+        if ((rc = check_cuda(ctx, cudaMalloc(&ctx->d_part_idx, need * sizeof(int32_t)), "cudaMalloc(partial ids)"))) return rc;
+        ctx->part_capacity = need;
+    }
+    float* mean = ctx->d_colsum + (size_t)n_slabs * d;
+    const __nv_bfloat16* W = (const __nv_bfloat16*)ctx->unembed;
+    unigram_colsum_kernel<<<dim3((d + 127) / 128, n_slabs), 128, 0, st>>>(W, V, d, ctx->d_colsum);
+    unigram_mean_kernel<<<(d + 127) / 128, 128, 0, st>>>(ctx->d_colsum, n_slabs, V, d, mean);
+    unigram_centre_kernel<<<ctx->num_sms * 8, 256, 0, st>>>(W, mean, n, d, (__nv_bfloat16*)ctx->d_centred);
+    const CUtensorMap* tmE;
+    if ((rc = w_map(ctx, sh, &tmE, true))) return rc;
+    CUtensorMap tmA;
+    if ((rc = make_tensor_map(ctx, &tmA, ctx->d_centred, V, d, sh.a_box_rows))) return rc;
+    GemmParams p;
+    fill_common(ctx, p, V, sh);
+    p.part_val = ctx->d_part_val;
+    head_gemm_kernel<MODE_SUMSQ, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmE, p);
+    unigram_sum_kernel<<<(V + 255) / 256, 256, 0, st>>>(ctx->d_part_val, sh.n_chunks, V, d_dist2);
+    ctx->launches += 5;
+    if (k_uni > 0) {
+        unigram_smallest_k_kernel<<<1, 1024, 0, st>>>(d_dist2, V, k_uni, d_uni_idx);
+        ctx->launches += 1;
+    }
+    return check_cuda(ctx, cudaGetLastError(), "build_model_unigram launch");
 }
 
 }  // namespace ngs

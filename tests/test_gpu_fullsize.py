@@ -61,6 +61,17 @@ def test_model_table_sampled_rows(heads, name):
     assert np.array_equal(ext[sel], ref[sel])
 
 
+def test_model_unigram_sampled_rows_at_full_size(heads):
+    c, h = heads("C2")
+    idx, dist2 = h["ctx"].build_model_unigram(25)
+    dist2 = dist2.cpu().numpy().astype(np.float64)
+    rows = sample_rows(c["V"], 12, seed=11)
+    ref = oracle.unigram_dist2(h["W"], h["E"], rows=rows)
+    assert np.abs(dist2[rows] - ref).max() <= 2e-3 * ref.max()
+    assert np.array_equal(idx.cpu().numpy(), oracle.smallest_k(dist2, 25))       # integer stage: exact
+    assert np.isfinite(dist2).all() and (dist2 >= 0).all()
+
+
 @pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5"])
 def test_whole_step_at_full_size(heads, name):
     c, h = heads(name)
