@@ -625,15 +625,16 @@ static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks) {
         double best = -1.0;
         for (int g = std::min(16, n_mtiles); g >= 1; --g) {
             const int slots = sms / g, groups = (n_mtiles + g - 1) / g;
-            const double busy = (double)n_mtiles / (groups * g) * (double)(slots * g) / sms * (1.0 - 0.005 * (16 - g));
+            const double busy = (double)n_mtiles / (groups * g) * (double)(slots * g) / sms * (1.0 - 0.02 * (16 - g));
             if (busy > best + 1e-9) {
                 best = busy;
                 sh.group = g;
             }
         }
         const int slots = sms / sh.group;
-        // 256-row boxes need one TMA issue per k-block; fall back to smaller boxes only when the
-        // vocabulary is too small to give every slot a chunk
+        // 256-row boxes need one TMA issue per k-block and measured faster than better balanced chunks
+        // of smaller boxes; fall back to smaller boxes only when the vocabulary is too small to give
+        // every slot a chunk
         sh.box_n = 256;
         while (sh.box_n > 32 && (V + sh.box_n - 1) / sh.box_n < slots) sh.box_n >>= 1;
         const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
