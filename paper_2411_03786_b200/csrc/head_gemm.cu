@@ -65,6 +65,7 @@ struct GemmParams {
     int a_bytes;      // shared-memory bytes reserved for the A tile of a stage (multiple of 1024)
     int stage_bytes;  // a_bytes + boxes per tile * box bytes
     int stages;       // depth of the operand ring
+    int dual;         // 1: A has two m-tiles and every CTA computes both against its W slice (argmax only)
     unsigned long long* keys;
     unsigned int* ticket;
     int32_t* argmax;
@@ -301,7 +302,8 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
-            const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2;
+            const bool dual = MODE == MODE_ARGMAX && p.dual;
+            const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2 * (dual ? 2u : 1u);
             // W is a constant of the model: fill the ring with its tiles before waiting for the kernel
             // that produces the activations, then add the A tiles of those stages.
             int n_pref = 0;
@@ -326,6 +328,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + j) * BOX_N, full);
                 }
                 tma_load_2d(sa, &tmA, cur.kb * BLOCK_K, cur.un.m_tile * BLOCK_M, full);
+                if (dual) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * BLOCK_K, BLOCK_M, full);  // second m-tile
                 ++issued;
                 if (++stage == STAGES) {
                     stage = 0;
@@ -359,7 +362,9 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             while (ok && it.next(p, un)) {
                 for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
                     const int nb = min(MAX_BOXES, un.box_end - b0);
-                    const uint32_t as = tile & 1u, aphase = (tile >> 1) & 1u;
+                    // dual: the tile takes both accumulator stages (one per m-tile), so tiles do not overlap
+                    const bool dual = MODE == MODE_ARGMAX && p.dual;
+                    const uint32_t as = dual ? 0u : (tile & 1u), aphase = dual ? (tile & 1u) : ((tile >> 1) & 1u);
                     if (!mbar_wait(bar_tempty + 8 * as, aphase ^ 1u, abort_flag)) {
                         ok = false;
                         break;
@@ -379,6 +384,12 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                         for (int k = 0; k < BLOCK_K / 16; ++k)  // +32 bytes (2 x 16 B) per K = 16 slice
                             tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        if (dual) {  // the same W tile against the second m-tile, into the other accumulator
+                            const uint64_t adesc2 = make_kmajor_sw128_desc(sa + A_TILE_BYTES);
+#pragma unroll
+                            for (int k = 0; k < BLOCK_K / 16; ++k)
+                                tc_mma_bf16(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
                         tc_commit(bar_empty + 8 * stage);  // frees the stage once these MMAs have read it
                         if (++stage == STAGES) {
                             stage = 0;
@@ -404,6 +415,9 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // running reduction of this row over the unit's columns
             float best_v = MODE == MODE_SUMSQ ? 0.0f : -INFINITY;
             int best_i = 0x7FFFFFFF;
+            const bool dual = MODE == MODE_ARGMAX && p.dual;
+            float best_v2 = -INFINITY;  // dual: the row of the second m-tile on this lane
+            int best_i2 = 0x7FFFFFFF;
             // Sorted list, value descending, statically indexed so it stays in registers.  The k_tab live
             // entries sit at the bottom [KT - k_tab, KT); the slots above hold +inf, which nothing beats,
             // so the running threshold is always the last slot.
@@ -417,7 +431,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
                 const int nb = min(MAX_BOXES, un.box_end - b0);
-                const uint32_t as = tile & 1u, aphase = (tile >> 1) & 1u;
+                const uint32_t as = dual ? 0u : (tile & 1u), aphase = dual ? (tile & 1u) : ((tile >> 1) & 1u);
                 if (!mbar_wait(bar_tfull + 8 * as, aphase, abort_flag)) {
                     ok = false;
                     break;
@@ -480,11 +494,34 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                     }
                 }
+                if (dual) {
+                    for (int c = 0; c * 32 < n_valid; ++c) {
+                        uint32_t r[32];
+                        __syncwarp();
+                        tmem_ld32(lane_base + ACC_COLS + c * 32, r);
+                        tmem_wait_ld();
+                        const int cbase = col0 + c * 32;
+                        const int lim = n_valid - c * 32;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float v = __uint_as_float(r[j]);
+                            if (j < lim && v > best_v2) {
+                                best_v2 = v;
+                                best_i2 = cbase + j;
+                            }
+                        }
+                    }
+                }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * as);
             }
             if (!ok) break;
+            if (dual && row + BLOCK_M < p.a_rows) {
+                const unsigned long long key =
+                    ((unsigned long long)orderable_f32(best_v2) << 32) | (unsigned long long)(~(uint32_t)best_i2);
+                atomicMax(p.keys + row + BLOCK_M, key);
+            }
             if (row < p.a_rows) {
                 if (MODE == MODE_ARGMAX) {
                     const unsigned long long key =
@@ -586,22 +623,22 @@ __global__ void extend_table_kernel(const int32_t* __restrict__ tab, int V, int 
 // ------------------------------------------------------------------------------------------ host: unit shapes
 struct Shape {
     int box_n, box_idx, group, n_groups, n_slots, n_chunks, grid;
-    int a_box_rows, a_bytes, stage_bytes, stages, smem;
+    int a_box_rows, a_bytes, stage_bytes, stages, smem, dual;
 };
 
 // Derives the shared-memory geometry from (box_n, group, n_chunks, grid).
 static void finish_shape(Shape& sh, int a_rows, int V) {
     const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
     sh.box_idx = sh.box_n == 16 ? 0 : sh.box_n == 32 ? 1 : sh.box_n == 64 ? 2 : sh.box_n == 128 ? 3 : 4;
-    sh.n_groups = (n_mtiles + sh.group - 1) / sh.group;
+    sh.n_groups = sh.dual ? 1 : (n_mtiles + sh.group - 1) / sh.group;
     sh.n_slots = sh.grid / sh.group;
     const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
     const int chunk_max = (n_boxes + sh.n_chunks - 1) / sh.n_chunks;
     const int nb_max = std::min(TILE_N / sh.box_n, chunk_max);
     sh.a_box_rows = n_mtiles == 1 ? std::min(BLOCK_M, (a_rows + 7) / 8 * 8) : BLOCK_M;
-    sh.a_bytes = (sh.a_box_rows * BLOCK_K * 2 + 1023) / 1024 * 1024;
+    sh.a_bytes = sh.dual ? 2 * A_TILE_BYTES : (sh.a_box_rows * BLOCK_K * 2 + 1023) / 1024 * 1024;
     sh.stage_bytes = sh.a_bytes + (nb_max * sh.box_n * BLOCK_K * 2 + 1023) / 1024 * 1024;
-    const int pad = A_TILE_BYTES - sh.a_bytes;
+    const int pad = sh.dual ? 0 : A_TILE_BYTES - sh.a_bytes;
     sh.stages = std::min(MAX_STAGES, (SMEM_LIMIT - SMEM_MISC - pad) / sh.stage_bytes);
     sh.smem = sh.stages * sh.stage_bytes + pad + SMEM_MISC;
 }
@@ -611,10 +648,12 @@ static void finish_shape(Shape& sh, int a_rows, int V) {
 // share each W chunk, W is loaded in 256-row boxes (one TMA issue per k-block) and every slot
 // sweeps one chunk per m-group.  (Measured on B200, V=32000, d=4096: 32-row boxes 0.9, 64-row
 // 1.1, 256-row 1.2 PFLOP/s; groups of 8..16 beat groups of 2..4 by 10-20%.)
-static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks) {
+static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks, bool allow_dual) {
     const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
     Shape sh{};
-    if (n_mtiles == 1) {
+    if (n_mtiles == 1 || (n_mtiles == 2 && allow_dual)) {
+        // (two m-tiles: still one pass over W, every CTA computes both tiles against its slice)
+        sh.dual = n_mtiles == 2 ? 1 : 0;
         sh.box_n = 32;
         sh.group = 1;
         sh.n_chunks = (int)std::min<size_t>((size_t)std::min(sms, (V + 31) / 32), max_chunks);
@@ -645,7 +684,7 @@ static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks) {
     return sh;
 }
 
-static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks) {
+static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks, bool allow_dual = false) {
     // Tuning aid: NGRAM_SPEC_SHAPE="box,group,chunks" overrides the choice (values are clamped).
     if (const char* ov = getenv("NGRAM_SPEC_SHAPE")) {
         int box = 32, g = 1, c = 1;
@@ -661,15 +700,15 @@ static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks) {
             return s;
         }
     }
-    static std::map<std::tuple<int, int, int, int, size_t>, Shape> cache;
-    const auto key = std::make_tuple(a_rows, ctx->V, ctx->d, ctx->num_sms, max_chunks);
+    static std::map<std::tuple<int, int, int, int, size_t, bool>, Shape> cache;
+    const auto key = std::make_tuple(a_rows, ctx->V, ctx->d, ctx->num_sms, max_chunks, allow_dual);
     auto it = cache.find(key);
     if (it != cache.end()) return it->second;
-    Shape s = choose_shape(a_rows, ctx->V, ctx->num_sms, max_chunks);
+    Shape s = choose_shape(a_rows, ctx->V, ctx->num_sms, max_chunks, allow_dual);
     cache[key] = s;
     if (getenv("NGRAM_SPEC_TRACE"))
-        fprintf(stderr, "[ngram_spec] rows=%d V=%d d=%d: box=%d group=%d slots=%d chunks=%d grid=%d a_box=%d stages=%d stage=%dB smem=%dB\n",
-                a_rows, ctx->V, ctx->d, s.box_n, s.group, s.n_slots, s.n_chunks, s.grid, s.a_box_rows, s.stages, s.stage_bytes, s.smem);
+        fprintf(stderr, "[ngram_spec] rows=%d V=%d d=%d: dual=%d box=%d group=%d slots=%d chunks=%d grid=%d a_box=%d stages=%d stage=%dB smem=%dB\n",
+                a_rows, ctx->V, ctx->d, s.dual, s.box_n, s.group, s.n_slots, s.n_chunks, s.grid, s.a_box_rows, s.stages, s.stage_bytes, s.smem);
     return s;
 }
 
@@ -702,7 +741,8 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.a_rows = a_rows;
     p.V = ctx->V;
     p.num_kb = (ctx->d + BLOCK_K - 1) / BLOCK_K;
-    p.n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
+    p.n_mtiles = sh.dual ? 1 : (a_rows + BLOCK_M - 1) / BLOCK_M;  // dual: one unit covers both m-tiles
+    p.dual = sh.dual;
     p.box_n = sh.box_n;
     p.n_boxes = (ctx->V + sh.box_n - 1) / sh.box_n;
     p.n_chunks = sh.n_chunks;
@@ -727,7 +767,7 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
 int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st) {
     int rc = set_smem_attr<MODE_ARGMAX, 1>(ctx);
     if (rc) return rc;
-    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20);
+    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
     const CUtensorMap* tmW;
     if ((rc = w_map(ctx, sh, &tmW))) return rc;
     CUtensorMap tmA;
