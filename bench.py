@@ -467,6 +467,15 @@ def main():
             sec, acc_cpu, threads, sample, sampled = oracle_step_time(c, hist_h, lens_h, T_h, H_bits, W_bits, args.cpu_budget)
             cpu = {"value": acc_cpu / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
                    "s_per_step": sec}
+            if table:
+                # the oracle's table build on a row sample, projected to all V rows (each row costs 2 V d flop)
+                import oracle
+                n_rows = 2 * threads
+                t0 = time.perf_counter()
+                oracle.model_table(bf16_bits(E), W_bits, c["k_tab"], rows=np.linspace(0, c["V"] - 1, n_rows).astype(np.int64))
+                dt = time.perf_counter() - t0
+                cpu["table_build"] = {"rows_per_s": n_rows / dt, "projected_s": dt / n_rows * c["V"],
+                                      "sample": f"{n_rows} of {c['V']} rows"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16", "data": "synthetic", "config": cfg,
