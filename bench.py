@@ -223,6 +223,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU work for the oracle baseline")
     ap.add_argument("--no-table", action="store_true", help="skip timing the one-off table build")
     ap.add_argument("--scaled", action="store_true", help="also time draft/accept on bandwidth-sized batches")
+    ap.add_argument("--fuse", action="store_true", help="use verify_accept_commit (one launch) instead of the two calls")
     ap.add_argument("--no-graph", action="store_true", help="launch the step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -301,6 +302,8 @@ def main():
     out_a = (torch.empty(S, dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
              torch.empty((S, w + 1), dtype=torch.int32, device=dev))
 
+    fused = args.fuse      # measured equal on B200: dependent launch already hides the accept launch
+
     def step(timers=None):
         lens.copy_(lens0)                      # every iteration sees the same history length
         if timers:
@@ -308,12 +311,15 @@ def main():
         ctx.draft_context_ngrams(hist, lens, c["qs"], c["topk"], B, w, out=out_d)
         if timers:
             timers[1].record()
-        ctx.verify_lmhead_argmax(dH, out=out_v)
-        if timers:
-            timers[2].record()
-        ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), hist, lens, out=out_a)
-        if timers:
-            timers[3].record()
+        if timers or not fused:
+            ctx.verify_lmhead_argmax(dH, out=out_v)
+            if timers:
+                timers[2].record()
+            ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), hist, lens, out=out_a)
+            if timers:
+                timers[3].record()
+        else:   # verify + accept in one launch (the per-phase timing loop keeps them apart)
+            ctx.verify_accept_commit(dH, out_d[0], out_d[1], hist, lens, argmax=out_v[0], out=out_a)
 
     def barrier():
         if dist is not None:
@@ -332,7 +338,7 @@ def main():
         with torch.cuda.graph(graph, stream=side):
             step()
     run_step = graph.replay if graph is not None else step
-    launches_per_step = 3                      # draft, verify, accept (the length reset is a torch copy)
+    launches_per_step = 2 if (fused and S <= 256) else 3   # draft, verify(+accept) (the length reset is a torch copy)
 
     for _ in range(args.warmup):
         run_step()
@@ -402,8 +408,11 @@ def main():
         d_tok.copy_(h_tok, non_blocking=True)
         ctx.draft_context_ngrams(d_hist2, d_lens2, c["qs"], c["topk"], B, w, out=out_d)
         main.wait_stream(copy_stream)
-        ctx.verify_lmhead_argmax(d_H2, out=out_v)
-        ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), d_hist2, d_lens2, out=out_a2)
+        if fused:
+            ctx.verify_accept_commit(d_H2, out_d[0], out_d[1], d_hist2, d_lens2, argmax=out_v[0], out=out_a2)
+        else:
+            ctx.verify_lmhead_argmax(d_H2, out=out_v)
+            ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), d_hist2, d_lens2, out=out_a2)
         h_out.copy_(d_out, non_blocking=True)
 
     e2e_graph = None

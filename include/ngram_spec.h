@@ -157,6 +157,16 @@ int accept_and_commit(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_n
                       int32_t* d_best_row, int32_t* d_committed, void* stream);
 
 /*
+ * verify_lmhead_argmax followed by accept_and_commit as one call (Section 4.1 step iii plus the
+ * acceptance rule above).  M = S*B*(w+1) rows of hidden states.  For up to 256 sequences the CTA
+ * that merges the per-slice arg maxima also accepts and commits, so the step needs one launch
+ * less; larger batches run the two kernels back to back.  Arguments as in the two calls.
+ */
+int verify_accept_commit(spec_ctx* ctx, const void* d_hidden, const int32_t* d_drafts, const int32_t* d_ndrafts, int S,
+                         int B, int w, int32_t* d_argmax, int32_t* d_hist, int32_t* d_len, int cap,
+                         int32_t* d_acc_len, int32_t* d_best_row, int32_t* d_committed, void* stream);
+
+/*
  * Test aid: the same tensor-core main loop as the two head calls with a plain store epilogue.
  * d_logits[i, y] = <rows[i, :], unembed[y, :]> for i < m, as float32 [m, V].
  */

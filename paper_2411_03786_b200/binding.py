@@ -51,6 +51,8 @@ def load_library(build: bool = True) -> C.CDLL:
     lib.verify_lmhead_argmax.argtypes = [vp, vp, C.c_int, i32p, fp, vp]
     lib.accept_and_commit.argtypes = [vp, i32p, i32p, i32p, C.c_int, C.c_int, C.c_int, i32p, i32p, C.c_int, i32p,
                                       i32p, i32p, vp]
+    lib.verify_accept_commit.argtypes = [vp, vp, i32p, i32p, C.c_int, C.c_int, C.c_int, i32p, i32p, i32p, C.c_int, i32p,
+                                         i32p, i32p, vp]
     lib.spec_debug_logits.argtypes = [vp, vp, C.c_int, fp, vp]
     lib.verify_lmhead_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, i32p, fp, C.c_int, vp]
     lib.spec_launch_count.argtypes = [vp]
@@ -176,6 +178,23 @@ class SpecContext:
                                                 _ptr(lens, torch.int32), cap, _ptr(acc), _ptr(best), _ptr(com),
                                                 _stream()), "accept_and_commit")
         return acc, best, com
+
+    def verify_accept_commit(self, hidden, drafts, n_drafts, hist, lens, argmax=None, out=None):
+        """Fused verify + accept: returns ``(argmax[S, B, w+1], acc_len, best_row, committed)``."""
+        S, B, w = (int(x) for x in drafts.shape)
+        cap = int(hist.shape[1])
+        dev = hist.device
+        if argmax is None:
+            argmax = torch.empty(S * B * (w + 1), dtype=torch.int32, device=dev)
+        if out is None:
+            out = (torch.empty(S, dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+                   torch.empty((S, w + 1), dtype=torch.int32, device=dev))
+        acc, best, com = out
+        self._check(self._lib.verify_accept_commit(self._h, _ptr(hidden, torch.bfloat16), _ptr(drafts, torch.int32),
+                                                   _ptr(n_drafts, torch.int32), S, B, w, _ptr(argmax, torch.int32),
+                                                   _ptr(hist, torch.int32), _ptr(lens, torch.int32), cap, _ptr(acc),
+                                                   _ptr(best), _ptr(com), _stream()), "verify_accept_commit")
+        return argmax.view(S, B, w + 1), acc, best, com
 
     def debug_logits(self, rows: torch.Tensor) -> torch.Tensor:
         m = int(rows.shape[0])

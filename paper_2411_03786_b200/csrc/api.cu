@@ -4,6 +4,7 @@
 
 #include <cuda_bf16.h>
 
+#include "accept.cuh"
 #include "common.cuh"
 
 static char g_err[256] = "";
@@ -212,7 +213,30 @@ int verify_lmhead_argmax(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_
     if (M < 0 || M > SPEC_MAX_VERIFY_ROWS) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax: need 0 <= M <= %d", SPEC_MAX_VERIFY_ROWS);
     if (M == 0) return SPEC_OK;
     cudaSetDevice(ctx->device);
-    return launch_verify(ctx, d_hidden, M, d_argmax, d_max, (cudaStream_t)stream);
+    return launch_verify(ctx, d_hidden, M, d_argmax, d_max, (cudaStream_t)stream, nullptr);
+}
+
+int verify_accept_commit(spec_ctx* ctx, const void* d_hidden, const int32_t* d_drafts, const int32_t* d_ndrafts, int S, int B,
+                         int w, int32_t* d_argmax, int32_t* d_hist, int32_t* d_len, int cap, int32_t* d_acc_len,
+                         int32_t* d_best_row, int32_t* d_committed, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "verify_accept_commit: ctx is NULL");
+    if (!d_hidden || !d_drafts || !d_ndrafts || !d_argmax || !d_hist || !d_len || !d_acc_len || !d_best_row || !d_committed)
+        return fail(ctx, SPEC_ERR_ARG, "verify_accept_commit: NULL pointer");
+    if (!aligned16(d_hidden)) return fail(ctx, SPEC_ERR_ARG, "verify_accept_commit: d_hidden must be 16-byte aligned");
+    if (S < 0 || cap <= 0) return fail(ctx, SPEC_ERR_ARG, "verify_accept_commit: need S >= 0, cap > 0");
+    if (B < 1 || B > kMaxB || w < 1 || w > kMaxW) return fail(ctx, SPEC_ERR_ARG, "verify_accept_commit: need 1<=B<=%d, 1<=w<=%d", kMaxB, kMaxW);
+    const long long M = (long long)S * B * (w + 1);
+    if (M > SPEC_MAX_VERIFY_ROWS) return fail(ctx, SPEC_ERR_ARG, "verify_accept_commit: S*B*(w+1) exceeds %d rows", SPEC_MAX_VERIFY_ROWS);
+    if (S == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    if (S > 256) {  // many sequences: one warp per sequence in its own kernel is the faster way to accept
+        int rc = launch_verify(ctx, d_hidden, (int)M, d_argmax, nullptr, (cudaStream_t)stream, nullptr);
+        if (rc) return rc;
+        return launch_accept(ctx, d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row,
+                             d_committed, (cudaStream_t)stream);
+    }
+    const AcceptArgs q{d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row, d_committed, nullptr};
+    return launch_verify(ctx, d_hidden, (int)M, d_argmax, nullptr, (cudaStream_t)stream, &q);
 }
 
 int accept_and_commit(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_ndrafts, const int32_t* d_argmax, int S,

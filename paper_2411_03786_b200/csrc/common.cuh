@@ -115,7 +115,9 @@ bool aligned16(const void* p);
 int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows);
 
 // head_gemm.cu
-int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st);
+struct AcceptArgs;
+int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st,
+                  const AcceptArgs* fuse);
 int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
                  int32_t* d_ext, cudaStream_t st);
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st);

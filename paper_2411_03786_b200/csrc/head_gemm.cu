@@ -32,6 +32,7 @@
 #include <tuple>
 #include <vector>
 
+#include "accept.cuh"
 #include "common.cuh"
 
 namespace ngs {
@@ -75,6 +76,8 @@ struct GemmParams {
     int32_t* part_idx;
     float* logits;     // [a_rows, V]
     int* status;
+    int fuse_accept;   // argmax mode: the CTA that merges the keys also accepts and commits
+    AcceptArgs acc;
 };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
@@ -560,6 +563,12 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (p.maxv) p.maxv[i] = from_orderable_f32((uint32_t)(key >> 32));
                 }
                 if (et == 0) *p.ticket = 0u;
+                if (p.fuse_accept) {
+                    // the predictions are complete: greedy acceptance right here saves a kernel launch
+                    __threadfence();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    for (int sq = et >> 5; sq < p.acc.S; sq += 4) accept_sequence(p.acc, sq, lane);
+                }
             }
         }
     }
@@ -762,9 +771,12 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.part_idx = nullptr;
     p.logits = nullptr;
     p.status = ctx->d_status;
+    p.fuse_accept = 0;
+    p.acc = AcceptArgs{};
 }
 
-int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st) {
+int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st,
+                  const AcceptArgs* fuse) {
     int rc = set_smem_attr<MODE_ARGMAX, 1>(ctx);
     if (rc) return rc;
     const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
@@ -776,6 +788,11 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     fill_common(ctx, p, M, sh);
     p.argmax = d_argmax;
     p.maxv = d_max;
+    if (fuse) {
+        p.fuse_accept = 1;
+        p.acc = *fuse;
+        p.acc.status = ctx->d_status;
+    }
     cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, tmA, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax launch");
@@ -1043,7 +1060,7 @@ extern "C" int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d,
         if (e == cudaSuccess) e = cudaMemsetAsync(d_argmax, 0xFF, sizeof(int32_t) * (size_t)M, st);
         rc = check_cuda(&tmp, e, "verify_lmhead_argmax_noalloc: cudaMemsetAsync");
     }
-    if (rc == SPEC_OK) rc = launch_verify(&tmp, d_hidden, M, d_argmax, d_max, st);
+    if (rc == SPEC_OK) rc = launch_verify(&tmp, d_hidden, M, d_argmax, d_max, st, nullptr);
     if (rc != SPEC_OK) return fail(nullptr, rc, "%s", tmp.err);
     return SPEC_OK;
 }

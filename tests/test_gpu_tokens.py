@@ -172,3 +172,41 @@ def test_toy_model_decode_is_lossless_and_fully_accepted(ngs):
         assert accs == a2
     assert ctx.get_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("S,B,w", [(1, 8, 5), (7, 4, 3), (64, 16, 8), (300, 2, 2)])
+def test_fused_verify_accept_equals_the_two_calls_and_the_oracle(ngs, S, B, w):
+    V, d = 777, 96
+    g = np.random.default_rng(S * 100 + B)
+    W = synth.gaussian_weights(V, d, 1.0, 3, "W")
+    ctx = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
+    M = S * B * (w + 1)
+    drafts = g.integers(0, V, (S, B, w)).astype(np.int32)
+    nd = g.integers(0, B + 1, S).astype(np.int32)
+    targets = g.integers(0, V, (S, B, w + 1)).astype(np.int32)
+    for s in range(S):                                  # plant accepted prefixes of random length
+        b, a = int(g.integers(0, B)), int(g.integers(0, w + 1))
+        targets[s, b, :a] = drafts[s, b, :a]
+    H = synth.hidden_planted(W, targets.reshape(-1), seed=S, gain=24.0)
+    cap = 32
+    lens = g.integers(0, cap - 2, S).astype(np.int32)
+    lens[0] = cap - 1                                   # too full for more than one token
+    hist = np.full((S, cap), -1, np.int32)
+    for s in range(S):
+        hist[s, :lens[s]] = g.integers(0, V, lens[s])
+    dH, dD, dN = dev_bf16(H), dev_i32(drafts), dev_i32(nd)
+    h1, l1 = dev_i32(hist), dev_i32(lens)
+    am, _ = ctx.verify_lmhead_argmax(dH)
+    acc1, best1, com1 = ctx.accept_and_commit(dD, dN, am.view(S, B, w + 1), h1, l1)
+    h2, l2 = dev_i32(hist), dev_i32(lens)
+    am2, acc2, best2, com2 = ctx.verify_accept_commit(dH, dD, dN, h2, l2)
+    assert torch.equal(am2.reshape(-1), am) and np.array_equal(am.cpu().numpy(), targets.reshape(-1))
+    for a, b in ((acc1, acc2), (best1, best2), (com1, com2), (h1, h2), (l1, l2)):
+        assert torch.equal(a, b)
+    h_ref, l_ref = hist.copy(), lens.copy()
+    acc_r, best_r, com_r = oracle.accept_commit(drafts, nd, targets, h_ref, l_ref)
+    assert np.array_equal(acc2.cpu().numpy(), acc_r) and np.array_equal(best2.cpu().numpy(), best_r)
+    assert np.array_equal(com2.cpu().numpy(), com_r) and np.array_equal(h2.cpu().numpy(), h_ref)
+    assert np.array_equal(l2.cpu().numpy(), l_ref)
+    ctx.get_status()
+    ctx.close()
