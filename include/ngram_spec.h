@@ -25,6 +25,10 @@
  *     d % 8 == 0, M <= SPEC_MAX_VERIFY_ROWS, history length < 2^28.
  *   - Data errors found on the device (token out of range, history overflow, a bounded wait that
  *     expired) never trap: they set bits in a status word that spec_get_status returns.
+ *   - The step's kernels are launched with programmatic dependent launch: a kernel of this library
+ *     may be scheduled while the previous kernel of the stream is still running, but it waits for
+ *     that kernel to finish before it reads anything but the model weights.  Stream order is kept
+ *     for every buffer; other work enqueued before or after behaves as with ordinary launches.
  *   - The GPU must be compute capability 10.0 (sm_100a).  There is no CPU fallback: every entry
  *     point fails with SPEC_ERR_CUDA when no such device is usable.
  */
