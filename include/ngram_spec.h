@@ -61,6 +61,8 @@ enum {
 
 enum { SPEC_F32 = 0, SPEC_BF16 = 1 };
 enum { SPEC_FLAG_DEDUP = 1, SPEC_FLAG_MODEL_FILL = 2 };
+/* OR into the draft flags to reserve n (0..255) of the B draft rows for the model strategy */
+#define SPEC_FLAG_RESERVE(n) (((n) & 0xFF) << 8)
 enum { SPEC_MAX_VERIFY_ROWS = 65536 };
 enum { SPEC_NOALLOC_MAX_ROWS = 4096 }; /* row limit of verify_lmhead_argmax_noalloc */
 
@@ -124,7 +126,9 @@ int spec_set_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, con
  * descending, ties by the later occurrence; the first topk continuations become draft rows.
  * Rows are taken in qs order; with SPEC_FLAG_DEDUP a row equal to an earlier row is skipped; with
  * SPEC_FLAG_MODEL_FILL the remaining rows are the extended model bigram of the last token in rank
- * order.  Histories shorter than q+w give no rows for that q.
+ * order.  Histories shorter than q+w give no rows for that q.  SPEC_FLAG_RESERVE(n) caps the context
+ * rows at B - n so that n rows are left to the model strategy (the allocation between strategies is
+ * an open knob in the paper, Section 5.2); a model row is then compared with the rows taken only.
  *   qs         host array of n_q query lengths (n_q = 0: model rows only).
  *   d_drafts   [S, B, w] out, unused rows = -1.      d_ndrafts [S] out.
  *   d_src      [S, B] out or NULL: q of the producing strategy, 0 = model, -1 = unused.

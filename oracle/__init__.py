@@ -24,6 +24,11 @@ FLAG_DEDUP = 1
 FLAG_MODEL_FILL = 2
 
 
+def flag_reserve(n: int) -> int:
+    """Flag bits that reserve ``n`` draft rows for the model strategy."""
+    return (int(n) & 0xFF) << 8
+
+
 def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (OpenMP over independent rows / sequences)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):

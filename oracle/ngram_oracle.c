@@ -139,21 +139,25 @@ void oracle_extend_table(const int32_t* T, int V, int k_tab, int w, int32_t* ext
  * in the caller's priority order, at most topk rows each; then, if asked, the
  * extended model bigram of the last token in rank order.  With dedup a row equal
  * in all w tokens to one already taken is skipped.  Unused rows are -1.
- * flags: bit0 = dedup, bit1 = model fill.
+ * flags: bit0 = dedup, bit1 = model fill, bits 8..15 = rows reserved for the model strategy (the
+ * context strategies together take at most B minus that many rows; the paper leaves the
+ * allocation between strategies open, Section 5.2).
  * src[b] = q of the strategy that produced row b, 0 for the model, -1 unused.
  */
 int oracle_draft_sequence(const int32_t* hist, int L, const int* qs, int n_q, int topk, int B, int w,
                           int flags, const int32_t* T, int V, int k_tab,
                           int32_t* drafts, int32_t* src, int32_t* counts) {
     int dedup = flags & 1, model_fill = flags & 2;
+    int reserve = (flags >> 8) & 0xFF;
+    int ctx_cap = reserve >= B ? 0 : B - reserve;
     int n = 0;
     for (int i = 0; i < B * w; ++i) drafts[i] = -1;
     for (int b = 0; b < B; ++b) { src[b] = -1; counts[b] = 0; }
     int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > k_tab ? topk : k_tab) * (size_t)w);
     int32_t* cnt = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > 0 ? topk : 1));
-    for (int qi = 0; qi < n_q && n < B; ++qi) {
+    for (int qi = 0; qi < n_q && n < ctx_cap; ++qi) {
         int m = oracle_context_draft(hist, L, qs[qi], w, topk, cand, cnt, NULL);
-        for (int r = 0; r < m && n < B; ++r) {
+        for (int r = 0; r < m && n < ctx_cap; ++r) {
             int dup = 0;
             if (dedup)
                 for (int b = 0; b < n && !dup; ++b)

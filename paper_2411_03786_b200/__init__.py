@@ -6,8 +6,8 @@ no CPU path; importing works without a GPU (so the build can be checked), but cr
 ``SpecContext`` without an sm_100 device raises.
 """
 from .binding import (FLAG_DEDUP, FLAG_MODEL_FILL, STATUS_CAPACITY, STATUS_GROUPS, STATUS_TIMEOUT,
-                      STATUS_TOKEN_RANGE, SpecContext, SpecError, declared_symbols, load_library,
+                      STATUS_TOKEN_RANGE, SpecContext, SpecError, declared_symbols, flag_reserve, load_library,
                       verify_lmhead_argmax_noalloc)
 
-__all__ = ["SpecContext", "SpecError", "load_library", "declared_symbols", "verify_lmhead_argmax_noalloc", "FLAG_DEDUP", "FLAG_MODEL_FILL",
+__all__ = ["SpecContext", "SpecError", "load_library", "declared_symbols", "flag_reserve", "verify_lmhead_argmax_noalloc", "FLAG_DEDUP", "FLAG_MODEL_FILL",
            "STATUS_TOKEN_RANGE", "STATUS_CAPACITY", "STATUS_TIMEOUT", "STATUS_GROUPS"]

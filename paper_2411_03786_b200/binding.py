@@ -17,6 +17,11 @@ _HEADER = os.path.join(os.path.dirname(os.path.abspath(__file__)), "..", "includ
 _lib = None
 
 
+def flag_reserve(n: int) -> int:
+    """Draft flag bits that reserve ``n`` rows for the model strategy (SPEC_FLAG_RESERVE)."""
+    return (int(n) & 0xFF) << 8
+
+
 class SpecError(RuntimeError):
     pass
 

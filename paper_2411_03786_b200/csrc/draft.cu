@@ -383,7 +383,8 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     // ---- mixed allocation: context rows in query order, then model rows by rank; drop duplicates.
     // Candidate rows are gathered side by side, a row is a duplicate if any earlier candidate equals
     // it (equality is transitive, so this is the same as comparing with the rows already taken),
-    // and the first B survivors become the drafts.
+    // and the first B survivors become the drafts.  (With rows reserved for the model the
+    // comparison is staged: see below.)
     const bool dedup = (P.flags & SPEC_FLAG_DEDUP) != 0;
     if (tid == 0) {
         int off = 0;
@@ -421,13 +422,15 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         }
     }
     __syncthreads();
-    if (dedup) {
-        // all (earlier, later) pairs side by side; a later row equal to an earlier valid row is dropped
-        int32_t* dropped = sm->row_of_tmp;
+    // Rows reserved for the model strategy: the context strategies together take at most B - reserve.
+    const int reserve = min(P.B, (P.flags >> 8) & 0xFF);
+    const int n_ctx = sm->cand_off[P.n_q];
+    int32_t* dropped = sm->row_of_tmp;
+    // all (earlier, later) pairs in [pair_lo, pair_hi) side by side: a later row equal to an earlier live row is dropped
+    auto drop_duplicates = [&](int pair_lo, int pair_hi) {
         for (int i = tid; i < n_cand; i += nthr) dropped[i] = 0;
         __syncthreads();
-        const int n_pairs = n_cand * (n_cand - 1) / 2;
-        for (int pi = tid; pi < n_pairs; pi += nthr) {
+        for (int pi = pair_lo + tid; pi < pair_hi; pi += nthr) {
             // pair index -> (ci, j) with j < ci: ci is the largest integer with ci (ci - 1) / 2 <= pi
             int ci = (int)((1.0f + sqrtf(1.0f + 8.0f * (float)pi)) * 0.5f);
             while (ci * (ci - 1) / 2 > pi) --ci;
@@ -442,18 +445,48 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         for (int i = tid; i < n_cand; i += nthr)
             if (dropped[i]) sm->cand_keep[i] = 0;
         __syncthreads();
-    }
-    if (warp == 0) {
-        int base = 0;
-        for (int c0 = 0; c0 < n_cand; c0 += 32) {
+    };
+    // warp 0: live candidates in [c_lo, c_hi) get draft rows first_row, first_row + 1, ... below row_limit;
+    // the others are switched off.  Returns the next free row.
+    auto assign_rows = [&](int c_lo, int c_hi, int first_row, int row_limit) {
+        int base = first_row;
+        for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
             const int ci = c0 + lane;
-            const bool k = ci < n_cand && sm->cand_keep[ci] != 0;
+            const bool k = ci < c_hi && sm->cand_keep[ci] != 0;
             const unsigned mask = __ballot_sync(0xffffffffu, k);
             const int pos = base + __popc(mask & ((1u << lane) - 1u));
-            if (k && pos < P.B) sm->row_of[pos] = ci;
+            if (k) {
+                if (pos < row_limit) sm->row_of[pos] = ci;
+                else sm->cand_keep[ci] = 0;
+            }
             base += __popc(mask);
         }
-        if (lane == 0) sm->n_out = min(base, P.B);
+        return min(base, row_limit);
+    };
+    const int all_pairs = n_cand * (n_cand - 1) / 2;
+    if (reserve == 0) {
+        // a row is a duplicate if any earlier candidate equals it: the rows beyond B are never
+        // followed by a row that is taken, so comparing with every earlier candidate is exact
+        if (dedup) drop_duplicates(0, all_pairs);
+        if (warp == 0) {
+            const int n_rows = assign_rows(0, n_cand, 0, P.B);
+            if (lane == 0) sm->n_out = n_rows;
+        }
+    } else {
+        // context rows first, cut at B - reserve; model rows are then compared with the rows taken only
+        const int ctx_pairs = n_ctx * (n_ctx - 1) / 2;
+        if (dedup) drop_duplicates(0, ctx_pairs);
+        if (warp == 0) {
+            const int n_rows = assign_rows(0, n_ctx, 0, P.B - reserve);
+            if (lane == 0) sm->n_out = n_rows;
+        }
+        __syncthreads();
+        if (dedup) drop_duplicates(ctx_pairs, all_pairs);
+        if (warp == 0) {
+            const int n_rows = assign_rows(n_ctx, n_cand, sm->n_out, P.B);
+            __syncwarp();
+            if (lane == 0) sm->n_out = n_rows;
+        }
     }
     __syncthreads();
     const int n = sm->n_out;

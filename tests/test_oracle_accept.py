@@ -102,9 +102,10 @@ def test_no_drafts_commits_the_plain_greedy_token():
 def brute_mix(hist, qs, topk, B, w, flags, T):
     from test_oracle_context import brute_context
     rows, src, cnt = [], [], []
+    ctx_cap = max(0, B - ((flags >> 8) & 0xFF))
     for q in qs:
         for c, n, _ in brute_context(hist, q, w, topk):
-            if len(rows) == B:
+            if len(rows) >= ctx_cap:
                 break
             if (flags & 1) and list(c) in rows:
                 continue
@@ -134,7 +135,7 @@ def test_mixing_against_brute_force():
         n_q = int(g.integers(0, 4))
         qs = [int(q) for q in g.permutation([1, 2, 3, 4])[:n_q]]
         topk, B, w = int(g.integers(1, 5)), int(g.integers(1, 9)), int(g.integers(1, 5))
-        flags = int(g.integers(0, 4))
+        flags = int(g.integers(0, 4)) | (oracle.flag_reserve(int(g.integers(0, B + 2))) if trial % 3 == 0 else 0)
         cap = (L + 3) // 4 * 4 + 4
         h2 = np.full((1, cap), -1, np.int32)
         h2[0, :L] = hist
@@ -156,3 +157,19 @@ def test_context_rows_come_first_then_model_rows_in_rank_order():
     assert src[0].tolist() == [1, 0, 0, -1] and cnt[0].tolist() == [2, 0, 0, 0]
     drafts, nd, src, _ = oracle.draft_batch(hist, np.array([7], np.int32), [1], 2, 4, 2, 2, T)  # no dedup
     assert nd[0] == 4 and drafts[0].tolist() == [[1, 2], [1, 2], [2, 0], [0, 1]]
+
+
+def test_rows_reserved_for_the_model_cap_the_context_rows():
+    T = np.array([[1, 2, 0], [2, 0, 1], [0, 1, 2]], np.int32)
+    # after 0: (1,2) at 0, (2,1) at 3, (1,1) at 6, each once => ranked by recency: (1,1), (2,1), (1,2)
+    hist = np.array([[0, 1, 2, 0, 2, 1, 0, 1, 1, 0, -1, -1]], np.int32)
+    lens = np.array([10], np.int32)
+    d, nd, src, _ = oracle.draft_batch(hist, lens, [1], 4, 4, 2, 3, T)
+    assert nd[0] == 4 and src[0].tolist() == [1, 1, 1, 0]
+    assert d[0].tolist() == [[1, 1], [2, 1], [1, 2], [2, 0]]      # model rank 0 = (1,2) is a duplicate, rank 1 = (2,0)
+    d, nd, src, _ = oracle.draft_batch(hist, lens, [1], 4, 4, 2, 3 | oracle.flag_reserve(2), T)
+    assert nd[0] == 4 and src[0].tolist() == [1, 1, 0, 0]
+    # the context row (1,2) was cut by the reservation, so the model's (1,2) is not a duplicate of a row taken
+    assert d[0].tolist() == [[1, 1], [2, 1], [1, 2], [2, 0]]
+    d, nd, src, _ = oracle.draft_batch(hist, lens, [1], 4, 4, 2, 3 | oracle.flag_reserve(9), T)
+    assert src[0, :nd[0]].tolist() == [0] * int(nd[0])                        # everything reserved: model rows only
