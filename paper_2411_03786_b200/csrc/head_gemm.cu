@@ -30,7 +30,6 @@
 #include <algorithm>
 #include <map>
 #include <tuple>
-#include <vector>
 
 #include "accept.cuh"
 #include "common.cuh"
