@@ -60,7 +60,7 @@ enum {
 };
 
 enum { SPEC_F32 = 0, SPEC_BF16 = 1 };
-enum { SPEC_FLAG_DEDUP = 1, SPEC_FLAG_MODEL_FILL = 2 };
+enum { SPEC_FLAG_DEDUP = 1, SPEC_FLAG_MODEL_FILL = 2, SPEC_FLAG_KEY_NEXT_TOKEN = 4 };
 /* OR into the draft flags to reserve n (0..255) of the B draft rows for the model strategy */
 #define SPEC_FLAG_RESERVE(n) (((n) & 0xFF) << 8)
 enum { SPEC_MAX_VERIFY_ROWS = 65536 };
@@ -129,6 +129,8 @@ int spec_set_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, con
  * order.  Histories shorter than q+w give no rows for that q.  SPEC_FLAG_RESERVE(n) caps the context
  * rows at B - n so that n rows are left to the model strategy (the allocation between strategies is
  * an open knob in the paper, Section 5.2); a model row is then compared with the rows taken only.
+ * SPEC_FLAG_KEY_NEXT_TOKEN groups the matches by their next token only (counting "the tokens that
+ * follow each occurrence"); the row of a group is then the w tokens after its latest occurrence.
  *   qs         host array of n_q query lengths (n_q = 0: model rows only).
  *   d_drafts   [S, B, w] out, unused rows = -1.      d_ndrafts [S] out.
  *   d_src      [S, B] out or NULL: q of the producing strategy, 0 = model, -1 = unused.

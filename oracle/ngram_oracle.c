@@ -63,8 +63,19 @@ void oracle_round_to_bf16(const float* in, uint16_t* out, long n) {
  * Order: count descending, ties by the later occurrence (last descending).
  * Returns the number of rows written (<= topk).  rows is [topk, w].
  */
+int oracle_context_draft_keyed(const int32_t* hist, int L, int q, int w, int key_len, int topk,
+                               int32_t* rows, int32_t* counts, int32_t* lasts);
+
 int oracle_context_draft(const int32_t* hist, int L, int q, int w, int topk,
                          int32_t* rows, int32_t* counts, int32_t* lasts) {
+    return oracle_context_draft_keyed(hist, L, q, w, w, topk, rows, counts, lasts);
+}
+
+/* The same with matches grouped by the first key_len tokens of the continuation only (key_len = w is
+ * the paper's rule; key_len = 1 counts "the tokens that follow each occurrence", one at a time).  The
+ * row emitted for a group is the w tokens after its latest occurrence. */
+int oracle_context_draft_keyed(const int32_t* hist, int L, int q, int w, int key_len, int topk,
+                               int32_t* rows, int32_t* counts, int32_t* lasts) {
     if (q < 1 || w < 1 || topk < 1 || L < q + w) return 0;
     const int32_t* query = hist + (L - q);
     int n_windows = L - q - w + 1;
@@ -83,7 +94,7 @@ int oracle_context_draft(const int32_t* hist, int L, int q, int w, int topk,
         for (int j = 0; j < n_groups && g < 0; ++j) {
             const int32_t* cj = hist + g_first[j] + q;
             int same = 1;
-            for (int t = 0; t < w; ++t)
+            for (int t = 0; t < key_len; ++t)
                 if (c[t] != cj[t]) { same = 0; break; }
             if (same) g = j;
         }
@@ -139,7 +150,7 @@ void oracle_extend_table(const int32_t* T, int V, int k_tab, int w, int32_t* ext
  * in the caller's priority order, at most topk rows each; then, if asked, the
  * extended model bigram of the last token in rank order.  With dedup a row equal
  * in all w tokens to one already taken is skipped.  Unused rows are -1.
- * flags: bit0 = dedup, bit1 = model fill, bits 8..15 = rows reserved for the model strategy (the
+ * flags: bit0 = dedup, bit1 = model fill, bit2 = group matches by their next token only, bits 8..15 = rows reserved for the model strategy (the
  * context strategies together take at most B minus that many rows; the paper leaves the
  * allocation between strategies open, Section 5.2).
  * src[b] = q of the strategy that produced row b, 0 for the model, -1 unused.
@@ -156,7 +167,7 @@ int oracle_draft_sequence(const int32_t* hist, int L, const int* qs, int n_q, in
     int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > k_tab ? topk : k_tab) * (size_t)w);
     int32_t* cnt = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > 0 ? topk : 1));
     for (int qi = 0; qi < n_q && n < ctx_cap; ++qi) {
-        int m = oracle_context_draft(hist, L, qs[qi], w, topk, cand, cnt, NULL);
+        int m = oracle_context_draft_keyed(hist, L, qs[qi], w, (flags & 4) ? 1 : w, topk, cand, cnt, NULL);
         for (int r = 0; r < m && n < ctx_cap; ++r) {
             int dup = 0;
             if (dedup)

@@ -82,7 +82,7 @@ struct DraftSmem {
 };
 
 // Group the match whose continuation starts at p (query index qi).
-__device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int p, int qi, int w, uint32_t hsh,
+__device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int p, int qi, int key_len, uint32_t hsh,
                                              int slots, int max_groups, int* rep, int* cnt, int* last,
                                              int* grp_slot, DraftSmem* sm) {
     if (*((volatile int*)&sm->overflow)) return;  // this pass is void already: do not fill the table further
@@ -108,7 +108,7 @@ __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int 
         if ((cur >> 28) == qi) {
             const int rp = cur & 0x0FFFFFFF;
             bool same = true;
-            for (int t = 0; t < w; ++t)
+            for (int t = 0; t < key_len; ++t)
                 if (h[rp + t] != h[p + t]) {
                     same = false;
                     break;
@@ -198,6 +198,8 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
 
     // ---- context N-grams
     const int n_scan = L - w;  // token index x = p - 1 runs over [0, n_scan)
+    // continuation tokens that identify a group: all w (the paper's rule) or the next token only
+    const int key_len = (P.flags & SPEC_FLAG_KEY_NEXT_TOKEN) ? 1 : w;
     const int t0 = sm->tq[0], t1 = sm->tq[1], t2 = sm->tq[2], t3 = sm->tq[3];
     bool any_q = false;
     for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + w);
@@ -273,13 +275,13 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                         }
                         const int p = x + 1;
                         uint32_t hc = 0x9E3779B9u;
-                        for (int t = 0; t < w; ++t) hc = fmix32(hc ^ (uint32_t)h[p + t]) + 0x7F4A7C15u;
+                        for (int t = 0; t < key_len; ++t) hc = fmix32(hc ^ (uint32_t)h[p + t]) + 0x7F4A7C15u;
                         for (int qi = 0; qi < P.n_q; ++qi) {
                             const int q = P.qs[qi];
                             if (m < q || L < q + w) continue;
                             const uint32_t hq = fmix32(hc + (uint32_t)qi * 0x632BE5ABu);
                             if (R > 1 && (int)(fmix32(hq ^ 0xA511E9B3u) % (uint32_t)R) != r) continue;
-                            insert_match(h, p, qi, w, hq, P.slots, P.max_groups, lrep, lcnt, llast, lgrp_slot, lsm);
+                            insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, lrep, lcnt, llast, lgrp_slot, lsm);
                         }
                     }
                 }

@@ -52,7 +52,7 @@ def test_draft_matches_oracle_on_paper_shaped_histories(ngs, small_ctx, name):
     hist = np.where(hist >= 0, hist % V, -1).astype(np.int32)
     T = random_table(V, c["k_tab"], 3)
     ext = oracle.extend_table(T, c["w"])
-    for flags in (3, 1, 2, 0):
+    for flags in (3, 1, 2, 0, 7):
         want = oracle.draft_batch(hist, lens, c["qs"], c["topk"], c["B"], c["w"], flags, T)
         assert_draft_equal(run_draft(small_ctx, hist, lens, c["qs"], c["topk"], c["B"], c["w"], flags, T), want)
         assert_draft_equal(run_draft(small_ctx, hist, lens, c["qs"], c["topk"], c["B"], c["w"], flags, T, ext), want)
@@ -74,7 +74,7 @@ def test_draft_random_small_alphabets_and_ragged_lengths(ngs, small_ctx):
         n_q = int(g.integers(0, 5))
         qs = [int(q) for q in g.permutation([1, 2, 3, 4])[:n_q]]
         B = int(g.integers(1, 65)); w = int(g.integers(1, 17)); topk = int(g.integers(1, B + 1))
-        flags = int(g.integers(0, 4)) | (oracle.flag_reserve(int(g.integers(0, B + 2))) if trial % 2 else 0)
+        flags = int(g.integers(0, 8)) | (oracle.flag_reserve(int(g.integers(0, B + 2))) if trial % 2 else 0)
         want = oracle.draft_batch(hist, lens, qs, topk, B, w, flags, T)
         assert_draft_equal(run_draft(small_ctx, hist, lens, qs, topk, B, w, flags, T), want)
     assert small_ctx.get_status() == 0

@@ -99,12 +99,27 @@ def test_no_drafts_commits_the_plain_greedy_token():
 
 
 # ----------------------------------------------------------------------------- mixing (Section 4.3)
+def brute_context_next_token(hist, q, w, topk):
+    """Groups keyed by the next token only; the row comes from the latest occurrence."""
+    hist = [int(t) for t in hist]
+    L = len(hist)
+    if L < q + w:
+        return []
+    groups = {}
+    for i in range(L - q - w + 1):
+        if hist[i:i + q] == hist[L - q:]:
+            cnt, _ = groups.get(hist[i + q], (0, -1))
+            groups[hist[i + q]] = (cnt + 1, i)
+    order = sorted(groups.items(), key=lambda kv: (-kv[1][0], -kv[1][1]))[:topk]
+    return [(tuple(hist[last + q:last + q + w]), cnt, last) for _, (cnt, last) in order]
+
+
 def brute_mix(hist, qs, topk, B, w, flags, T):
     from test_oracle_context import brute_context
     rows, src, cnt = [], [], []
     ctx_cap = max(0, B - ((flags >> 8) & 0xFF))
     for q in qs:
-        for c, n, _ in brute_context(hist, q, w, topk):
+        for c, n, _ in (brute_context(hist, q, w, topk) if not flags & 4 else brute_context_next_token(hist, q, w, topk)):
             if len(rows) >= ctx_cap:
                 break
             if (flags & 1) and list(c) in rows:
@@ -135,7 +150,7 @@ def test_mixing_against_brute_force():
         n_q = int(g.integers(0, 4))
         qs = [int(q) for q in g.permutation([1, 2, 3, 4])[:n_q]]
         topk, B, w = int(g.integers(1, 5)), int(g.integers(1, 9)), int(g.integers(1, 5))
-        flags = int(g.integers(0, 4)) | (oracle.flag_reserve(int(g.integers(0, B + 2))) if trial % 3 == 0 else 0)
+        flags = int(g.integers(0, 8)) | (oracle.flag_reserve(int(g.integers(0, B + 2))) if trial % 3 == 0 else 0)
         cap = (L + 3) // 4 * 4 + 4
         h2 = np.full((1, cap), -1, np.int32)
         h2[0, :L] = hist

@@ -116,3 +116,31 @@ def test_later_occurrence_wins_ties_and_count_wins_over_recency():
     rows, counts, lasts = oracle.context_draft(np.array(hist, np.int32), 1, 1, 3)
     # after 4: 1 (x2, last 4), 2 (x2, last 8), 3 (x1, last 6); window 10 has no continuation
     assert rows.reshape(-1).tolist() == [2, 1, 3] and counts.tolist() == [2, 2, 1] and lasts.tolist() == [8, 4, 6]
+
+
+def test_next_token_keyed_variant():
+    g = np.random.default_rng(21)
+    for trial in range(100):
+        L, q, w = int(g.integers(0, 80)), int(g.integers(1, 4)), int(g.integers(1, 5))
+        hist = g.integers(0, 3, L).astype(np.int32)
+        rows, counts, lasts = oracle.context_draft(hist, q, w, 10, key_len=1)
+        if L < q + w:
+            assert len(rows) == 0
+            continue
+        # counts are the histogram of the token right after each eligible occurrence of the query
+        nxt, last = collections.Counter(), {}
+        for i in range(L - q - w + 1):
+            if (hist[i:i + q] == hist[L - q:]).all():
+                t = int(hist[i + q])
+                nxt[t] += 1
+                last[t] = i
+        order = sorted(nxt, key=lambda t: (-nxt[t], -last[t]))[:10]
+        assert [int(r[0]) for r in rows] == order
+        assert counts.tolist() == [nxt[t] for t in order] and lasts.tolist() == [last[t] for t in order]
+        for r, l in zip(rows, lasts):                         # the row is what followed the latest occurrence
+            assert r.tolist() == hist[l + q:l + q + w].tolist()
+    # with w = 1 the variant and the paper's rule coincide
+    hist = g.integers(0, 4, 60).astype(np.int32)
+    a = oracle.context_draft(hist, 1, 1, 8)
+    b = oracle.context_draft(hist, 1, 1, 8, key_len=1)
+    assert all(np.array_equal(x, y) for x, y in zip(a, b))
