@@ -144,6 +144,12 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     int* llast = cluster.map_shared_rank(last, 0);
     int* lgrp_slot = cluster.map_shared_rank(grp_slot, 0);
 
+    // barrier over all CTAs of the sequence (a plain CTA barrier when there is only one: much cheaper)
+    auto pass_sync = [&]() {
+        if (csize == 1) __syncthreads();
+        else cluster.sync();
+    };
+
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
     const int s = (int)blockIdx.x / csize;
@@ -222,7 +228,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                     sm->overflow = 0;
                 }
             }
-            cluster.sync();  // the leader's table is ready
+            pass_sync();  // the leader's table is ready
             // scan: 128-bit loads, four per thread in flight; positions holding the last token are
             // collected in a bit mask and handled one by one (they are rare)
             const int4* h4 = reinterpret_cast<const int4*>(h);
@@ -286,9 +292,9 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                     }
                 }
             }
-            cluster.sync();  // every CTA's matches are in the table
+            pass_sync();  // every CTA's matches are in the table
             const int ov = *((volatile int*)&lsm->overflow);
-            cluster.sync();  // every CTA has read the flag before the leader may reset it
+            pass_sync();  // every CTA has read the flag before the leader may reset it
             if (ov) {
                 overflowed = true;
                 break;
@@ -376,11 +382,6 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     }
     if (!leader) return;  // nobody reads a non-leader's shared memory, and no cluster barrier follows
     __syncthreads();
-    if (gave_up) {
-        if (tid < kMaxNQ) sm->n_run[tid] = 0;
-        if (tid == 0) atomicOr(P.status, SPEC_STATUS_GROUPS);
-    }
-    __syncthreads();
 
     // ---- mixed allocation: context rows in query order, then model rows by rank; drop duplicates.
     // Candidate rows are gathered side by side, a row is a duplicate if any earlier candidate equals
@@ -389,6 +390,10 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     // comparison is staged: see below.)
     const bool dedup = (P.flags & SPEC_FLAG_DEDUP) != 0;
     if (tid == 0) {
+        if (gave_up) {  // too many distinct continuations even for 1024 passes: no context rows, and say so
+            for (int li = 0; li < kMaxNQ; ++li) sm->n_run[li] = 0;
+            atomicOr(P.status, SPEC_STATUS_GROUPS);
+        }
         int off = 0;
         for (int li = 0; li < P.n_q; ++li) {
             sm->cand_off[li] = off;
@@ -421,6 +426,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             sm->cand_src[ci] = src;
             sm->cand_cnt[ci] = count;
             sm->cand_keep[ci] = keep;
+            sm->row_of_tmp[ci] = 0;  // duplicate flag
         }
     }
     __syncthreads();
@@ -429,9 +435,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     const int n_ctx = sm->cand_off[P.n_q];
     int32_t* dropped = sm->row_of_tmp;
     // all (earlier, later) pairs in [pair_lo, pair_hi) side by side: a later row equal to an earlier live row is dropped
-    auto drop_duplicates = [&](int pair_lo, int pair_hi) {
-        for (int i = tid; i < n_cand; i += nthr) dropped[i] = 0;
-        __syncthreads();
+    auto mark_duplicates = [&](int pair_lo, int pair_hi) {
         for (int pi = pair_lo + tid; pi < pair_hi; pi += nthr) {
             // pair index -> (ci, j) with j < ci: ci is the largest integer with ci (ci - 1) / 2 <= pi
             int ci = (int)((1.0f + sqrtf(1.0f + 8.0f * (float)pi)) * 0.5f);
@@ -444,9 +448,6 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             if (same) dropped[ci] = 1;
         }
         __syncthreads();
-        for (int i = tid; i < n_cand; i += nthr)
-            if (dropped[i]) sm->cand_keep[i] = 0;
-        __syncthreads();
     };
     // warp 0: live candidates in [c_lo, c_hi) get draft rows first_row, first_row + 1, ... below row_limit;
     // the others are switched off.  Returns the next free row.
@@ -454,13 +455,11 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         int base = first_row;
         for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
             const int ci = c0 + lane;
-            const bool k = ci < c_hi && sm->cand_keep[ci] != 0;
+            const bool k = ci < c_hi && sm->cand_keep[ci] != 0 && dropped[ci] == 0;
             const unsigned mask = __ballot_sync(0xffffffffu, k);
             const int pos = base + __popc(mask & ((1u << lane) - 1u));
-            if (k) {
-                if (pos < row_limit) sm->row_of[pos] = ci;
-                else sm->cand_keep[ci] = 0;
-            }
+            if (k && pos < row_limit) sm->row_of[pos] = ci;
+            else if (ci < c_hi) sm->cand_keep[ci] = 0;
             base += __popc(mask);
         }
         return min(base, row_limit);
@@ -469,7 +468,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     if (reserve == 0) {
         // a row is a duplicate if any earlier candidate equals it: the rows beyond B are never
         // followed by a row that is taken, so comparing with every earlier candidate is exact
-        if (dedup) drop_duplicates(0, all_pairs);
+        if (dedup) mark_duplicates(0, all_pairs);
         if (warp == 0) {
             const int n_rows = assign_rows(0, n_cand, 0, P.B);
             if (lane == 0) sm->n_out = n_rows;
@@ -477,13 +476,13 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     } else {
         // context rows first, cut at B - reserve; model rows are then compared with the rows taken only
         const int ctx_pairs = n_ctx * (n_ctx - 1) / 2;
-        if (dedup) drop_duplicates(0, ctx_pairs);
+        if (dedup) mark_duplicates(0, ctx_pairs);
         if (warp == 0) {
             const int n_rows = assign_rows(0, n_ctx, 0, P.B - reserve);
             if (lane == 0) sm->n_out = n_rows;
         }
         __syncthreads();
-        if (dedup) drop_duplicates(ctx_pairs, all_pairs);
+        if (dedup) mark_duplicates(ctx_pairs, all_pairs);
         if (warp == 0) {
             const int n_rows = assign_rows(n_ctx, n_cand, sm->n_out, P.B);
             __syncwarp();
