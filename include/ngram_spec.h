@@ -177,6 +177,18 @@ int verify_accept_commit(spec_ctx* ctx, const void* d_hidden, const int32_t* d_d
                          int32_t* d_acc_len, int32_t* d_best_row, int32_t* d_committed, void* stream);
 
 /*
+ * Verification with the vocabulary sharded over several GPUs (one context per shard, each holding
+ * V_local rows of the unembedding that start at token id vocab_offset).  verify_lmhead_keys leaves,
+ * per row, a 64-bit key that orders as a signed integer by (logit, then lower global token id); the
+ * caller takes the element-wise maximum over the shards (e.g. an NCCL all-reduce with max on int64)
+ * and spec_unpack_keys turns the result into token ids and logits.  The paper runs on one GPU
+ * (Section 5); this is the natural split of its verification call for a head that is sharded.
+ *   d_keys [M] int64 out / in.   V_total = full vocabulary size (ids are clamped to it).
+ */
+int verify_lmhead_keys(spec_ctx* ctx, const void* d_hidden, int M, int vocab_offset, long long* d_keys, void* stream);
+int spec_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_argmax, float* d_max, void* stream);
+
+/*
  * Test aid: the same tensor-core main loop as the two head calls with a plain store epilogue.
  * d_logits[i, y] = <rows[i, :], unembed[y, :]> for i < m, as float32 [m, V].
  */

@@ -58,6 +58,8 @@ def load_library(build: bool = True) -> C.CDLL:
                                       i32p, i32p, vp]
     lib.verify_accept_commit.argtypes = [vp, vp, i32p, i32p, C.c_int, C.c_int, C.c_int, i32p, i32p, i32p, C.c_int, i32p,
                                          i32p, i32p, vp]
+    lib.verify_lmhead_keys.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp]
+    lib.spec_unpack_keys.argtypes = [vp, C.c_int, C.c_int, i32p, fp, vp]
     lib.spec_debug_logits.argtypes = [vp, vp, C.c_int, fp, vp]
     lib.verify_lmhead_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, i32p, fp, C.c_int, vp]
     lib.spec_launch_count.argtypes = [vp]
@@ -201,6 +203,15 @@ class SpecContext:
                                                    _ptr(best), _ptr(com), _stream()), "verify_accept_commit")
         return argmax.view(S, B, w + 1), acc, best, com
 
+    def verify_lmhead_keys(self, hidden: torch.Tensor, vocab_offset: int, keys: torch.Tensor | None = None):
+        """Per-row (logit, global id) keys of this context's vocabulary shard, as sortable int64."""
+        M = int(hidden.shape[0])
+        if keys is None:
+            keys = torch.empty(M, dtype=torch.int64, device=hidden.device)
+        self._check(self._lib.verify_lmhead_keys(self._h, _ptr(hidden, torch.bfloat16), M, int(vocab_offset),
+                                                 _ptr(keys, torch.int64), _stream()), "verify_lmhead_keys")
+        return keys
+
     def debug_logits(self, rows: torch.Tensor) -> torch.Tensor:
         m = int(rows.shape[0])
         out = torch.empty((m, self.V), dtype=torch.float32, device=rows.device)
@@ -224,4 +235,16 @@ def verify_lmhead_argmax_noalloc(unembed: torch.Tensor, hidden: torch.Tensor, ou
                                           _stream())
     if rc != 0:
         raise SpecError(f"verify_lmhead_argmax_noalloc failed ({rc}): {lib.spec_last_error(None).decode()}")
+    return am, mx
+
+
+def unpack_keys(keys: torch.Tensor, V_total: int, with_max: bool = False):
+    """Token ids (and winning logits) from merged shard keys."""
+    lib = load_library()
+    M = int(keys.shape[0])
+    am = torch.empty(M, dtype=torch.int32, device=keys.device)
+    mx = torch.empty(M, dtype=torch.float32, device=keys.device) if with_max else None
+    rc = lib.spec_unpack_keys(_ptr(keys, torch.int64), M, int(V_total), _ptr(am), _ptr(mx), _stream())
+    if rc != 0:
+        raise SpecError(f"spec_unpack_keys failed ({rc}): {lib.spec_last_error(None).decode()}")
     return am, mx

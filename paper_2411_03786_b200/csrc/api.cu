@@ -213,7 +213,7 @@ int verify_lmhead_argmax(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_
     if (M < 0 || M > SPEC_MAX_VERIFY_ROWS) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax: need 0 <= M <= %d", SPEC_MAX_VERIFY_ROWS);
     if (M == 0) return SPEC_OK;
     cudaSetDevice(ctx->device);
-    return launch_verify(ctx, d_hidden, M, d_argmax, d_max, (cudaStream_t)stream, nullptr);
+    return launch_verify(ctx, d_hidden, M, d_argmax, d_max, (cudaStream_t)stream, nullptr, nullptr, 0);
 }
 
 int verify_accept_commit(spec_ctx* ctx, const void* d_hidden, const int32_t* d_drafts, const int32_t* d_ndrafts, int S, int B,
@@ -230,13 +230,13 @@ int verify_accept_commit(spec_ctx* ctx, const void* d_hidden, const int32_t* d_d
     if (S == 0) return SPEC_OK;
     cudaSetDevice(ctx->device);
     if (S > 256) {  // many sequences: one warp per sequence in its own kernel is the faster way to accept
-        int rc = launch_verify(ctx, d_hidden, (int)M, d_argmax, nullptr, (cudaStream_t)stream, nullptr);
+        int rc = launch_verify(ctx, d_hidden, (int)M, d_argmax, nullptr, (cudaStream_t)stream, nullptr, nullptr, 0);
         if (rc) return rc;
         return launch_accept(ctx, d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row,
                              d_committed, (cudaStream_t)stream);
     }
     const AcceptArgs q{d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row, d_committed, nullptr};
-    return launch_verify(ctx, d_hidden, (int)M, d_argmax, nullptr, (cudaStream_t)stream, &q);
+    return launch_verify(ctx, d_hidden, (int)M, d_argmax, nullptr, (cudaStream_t)stream, &q, nullptr, 0);
 }
 
 int accept_and_commit(spec_ctx* ctx, const int32_t* d_drafts, const int32_t* d_ndrafts, const int32_t* d_argmax, int S,
@@ -260,6 +260,24 @@ int build_model_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_d
         return fail(ctx, SPEC_ERR_ARG, "build_model_unigram: need 0 <= k_uni <= min(1024, V) and d_uni_idx for k_uni > 0");
     cudaSetDevice(ctx->device);
     return launch_unigram(ctx, k_uni, d_uni_idx, d_dist2, (cudaStream_t)stream);
+}
+
+int verify_lmhead_keys(spec_ctx* ctx, const void* d_hidden, int M, int vocab_offset, long long* d_keys, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_keys: ctx is NULL");
+    if (!d_hidden || !d_keys) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_keys: NULL pointer");
+    if (!aligned16(d_hidden)) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_keys: d_hidden must be 16-byte aligned");
+    if (M < 0 || M > SPEC_MAX_VERIFY_ROWS) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_keys: need 0 <= M <= %d", SPEC_MAX_VERIFY_ROWS);
+    if (vocab_offset < 0 || (long long)vocab_offset + ctx->V > 0x7FFFFFFFll)
+        return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_keys: vocab_offset + V must fit in int32");
+    if (M == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    return launch_verify(ctx, d_hidden, M, nullptr, nullptr, (cudaStream_t)stream, nullptr, d_keys, vocab_offset);
+}
+
+int spec_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_argmax, float* d_max, void* stream) {
+    if (!d_keys || !d_argmax || M < 0 || V_total <= 0) return fail(nullptr, SPEC_ERR_ARG, "spec_unpack_keys: bad argument");
+    if (M == 0) return SPEC_OK;
+    return launch_unpack_keys(d_keys, M, V_total, d_argmax, d_max, (cudaStream_t)stream);
 }
 
 int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, void* stream) {

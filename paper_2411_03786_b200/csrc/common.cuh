@@ -117,7 +117,8 @@ int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, 
 // head_gemm.cu
 struct AcceptArgs;
 int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st,
-                  const AcceptArgs* fuse);
+                  const AcceptArgs* fuse, long long* d_keys_out, int idx_offset);
+int launch_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_argmax, float* d_max, cudaStream_t st);
 int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
                  int32_t* d_ext, cudaStream_t st);
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st);

@@ -77,6 +77,8 @@ struct GemmParams {
     int* status;
     int fuse_accept;   // argmax mode: the CTA that merges the keys also accepts and commits
     AcceptArgs acc;
+    long long* keys_out;  // argmax mode, vocabulary shard: export (value, id) keys instead of ids
+    int idx_offset;       // first token id of this shard
 };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
@@ -558,6 +560,13 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const unsigned long long key = atomicExch(p.keys + i, 0ull);
                     int idx = (int)(~(uint32_t)(key & 0xFFFFFFFFull));
                     if (idx < 0 || idx >= p.V) idx = 0;
+                    if (p.keys_out) {
+                        // shard of the vocabulary: global token id, and the sign bit flipped so that the key
+                        // orders correctly as a signed 64-bit integer (what a max all-reduce compares)
+                        const unsigned long long g = (key & 0xFFFFFFFF00000000ull) | (unsigned long long)(~(uint32_t)(idx + p.idx_offset));
+                        p.keys_out[i] = (long long)(g ^ 0x8000000000000000ull);
+                        continue;
+                    }
                     p.argmax[i] = idx;
                     if (p.maxv) p.maxv[i] = from_orderable_f32((uint32_t)(key >> 32));
                 }
@@ -772,10 +781,12 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.status = ctx->d_status;
     p.fuse_accept = 0;
     p.acc = AcceptArgs{};
+    p.keys_out = nullptr;
+    p.idx_offset = 0;
 }
 
 int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st,
-                  const AcceptArgs* fuse) {
+                  const AcceptArgs* fuse, long long* d_keys_out, int idx_offset) {
     int rc = set_smem_attr<MODE_ARGMAX, 1>(ctx);
     if (rc) return rc;
     const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
@@ -792,6 +803,8 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
         p.acc = *fuse;
         p.acc.status = ctx->d_status;
     }
+    p.keys_out = d_keys_out;
+    p.idx_offset = idx_offset;
     cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, tmA, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax launch");
@@ -861,6 +874,25 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
         if ((rc = check_cuda(ctx, cudaGetLastError(), "table extension launch"))) return rc;
     }
     return SPEC_OK;
+}
+
+// ------------------------------------------------------------------------------------------ vocabulary shards
+// Turns merged (value, id) keys (see keys_out above) back into token ids and winning logits.
+__global__ void unpack_keys_kernel(const long long* __restrict__ keys, int M, int V_total, int32_t* __restrict__ argmax,
+                                   float* __restrict__ maxv) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dependency_wait();
+    if (i >= M) return;
+    const unsigned long long key = (unsigned long long)keys[i] ^ 0x8000000000000000ull;
+    int idx = (int)(~(uint32_t)(key & 0xFFFFFFFFull));
+    if (idx < 0 || idx >= V_total) idx = 0;
+    argmax[i] = idx;
+    if (maxv) maxv[i] = from_orderable_f32((uint32_t)(key >> 32));
+}
+
+int launch_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_argmax, float* d_max, cudaStream_t st) {
+    cudaError_t e = launch_pdl(unpack_keys_kernel, dim3((M + 255) / 256), dim3(256), 0, st, d_keys, M, V_total, d_argmax, d_max);
+    return e == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------ model unigram
@@ -1059,7 +1091,7 @@ extern "C" int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d,
         if (e == cudaSuccess) e = cudaMemsetAsync(d_argmax, 0xFF, sizeof(int32_t) * (size_t)M, st);
         rc = check_cuda(&tmp, e, "verify_lmhead_argmax_noalloc: cudaMemsetAsync");
     }
-    if (rc == SPEC_OK) rc = launch_verify(&tmp, d_hidden, M, d_argmax, d_max, st, nullptr);
+    if (rc == SPEC_OK) rc = launch_verify(&tmp, d_hidden, M, d_argmax, d_max, st, nullptr, nullptr, 0);
     if (rc != SPEC_OK) return fail(nullptr, rc, "%s", tmp.err);
     return SPEC_OK;
 }

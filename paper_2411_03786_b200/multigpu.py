@@ -37,3 +37,37 @@ def whole_job_throughput(tokens_this_rank: float, ms_this_rank: float, device="c
     """``(tokens per second of the whole job, slowest rank's ms)``: all ranks' tokens over the slowest rank's time."""
     (ms,), (tokens,) = reduce_max_sum([ms_this_rank], [tokens_this_rank], device)
     return tokens / (ms / 1e3), ms
+
+
+def sharded_verify(ctx, hidden, vocab_offset: int, V_total: int, with_max: bool = False):
+    """Verification when every rank holds a slice of the vocabulary (``ctx`` was created with this
+    rank's rows of the unembedding, which start at token id ``vocab_offset``).
+
+    Each rank computes per-row (logit, id) keys over its slice; one all-reduce with MAX over the
+    int64 keys picks the winner across ranks (lowest global id on exact ties); the keys are then
+    unpacked.  Without a process group this is a single-shard verify.
+    """
+    import torch.distributed as dist
+    from .binding import unpack_keys
+    keys = ctx.verify_lmhead_keys(hidden, vocab_offset)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(keys, op=dist.ReduceOp.MAX)
+    return unpack_keys(keys, V_total, with_max)
+
+
+def pack_key(value: float, token_id: int) -> int:
+    """Host-side statement of the shard key format (for tests and debugging): a signed 64-bit integer
+    that is larger for a larger fp32 logit and, for equal logits, for a smaller token id."""
+    import struct
+    (u,) = struct.unpack("<I", struct.pack("<f", value))
+    u = (~u & 0xFFFFFFFF) if u & 0x80000000 else (u | 0x80000000)
+    k = ((u << 32) | (~token_id & 0xFFFFFFFF)) ^ 0x8000000000000000
+    return k - (1 << 64) if k >= (1 << 63) else k
+
+
+def unpack_key(key: int) -> tuple[float, int]:
+    import struct
+    k = (key + (1 << 64)) % (1 << 64) ^ 0x8000000000000000
+    u = k >> 32
+    u = (u & 0x7FFFFFFF) if u & 0x80000000 else (~u & 0xFFFFFFFF)
+    return struct.unpack("<f", struct.pack("<I", u))[0], (~k) & 0xFFFFFFFF

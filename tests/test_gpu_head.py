@@ -149,3 +149,33 @@ def test_model_unigram_matches_oracle(ngs, V, d, k):
         assert np.array_equal(idx, oracle.smallest_k(dist2, k))
     assert ctx.get_status() == 0
     ctx.close()
+
+
+def test_vocabulary_sharded_verify_equals_the_single_context(ngs):
+    """Three shard contexts on one GPU stand in for three ranks: keys per shard, element-wise max
+    (what the all-reduce computes), unpack."""
+    V, d, M = 3000, 192, 200
+    W = synth.gaussian_weights(V, d, d ** -0.5, 31, "W")
+    W[2500] = W[40]                     # an exact tie across shards: the lower global id must win
+    H = synth.hidden_literal(M, d, seed=32)
+    H[5] = W[40]
+    full = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
+    ref_am, ref_mx = full.verify_lmhead_argmax(dev_bf16(H), with_max=True)
+    bounds = [0, 1000, 1033, V]
+    keys = None
+    for lo, hi in zip(bounds[:-1], bounds[1:]):
+        Ws = dev_bf16(W[lo:hi])
+        shard = ngs.SpecContext(Ws, Ws)
+        k = shard.verify_lmhead_keys(dev_bf16(H), lo)
+        keys = k if keys is None else torch.maximum(keys, k)
+        torch.cuda.synchronize()
+        shard.close()
+    am, mx = ngs.unpack_keys(keys, V, with_max=True)
+    assert torch.equal(am, ref_am) and torch.equal(mx, ref_mx)
+    assert int(am[5]) == 40
+    from paper_2411_03786_b200 import multigpu
+    v, i = multigpu.unpack_key(int(keys[5]))
+    assert i == 40 and v == float(mx[5])
+    am2, _ = multigpu.sharded_verify(full, dev_bf16(H), 0, V)          # one shard, no process group
+    assert torch.equal(am2, ref_am)
+    full.close()

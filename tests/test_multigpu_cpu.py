@@ -57,3 +57,51 @@ def test_two_gloo_ranks_reduce_like_the_benchmark():
     for _, _, value, ms in res:
         assert ms == 20.0                                  # slowest rank
         assert abs(value - total / 0.020) < 1e-6           # whole-job tokens over the slowest rank's time
+
+
+def test_shard_keys_order_by_logit_then_lower_token_id():
+    vals = [-3.5, -0.0, 0.0, 1e-30, 2.25, 2.25, 1e30]
+    ids = [7, 3, 9, 1, 500, 20, 0]
+    keys = [multigpu.pack_key(v, i) for v, i in zip(vals, ids)]
+    for (v, i), k in zip(zip(vals, ids), keys):
+        v2, i2 = multigpu.unpack_key(k)
+        assert v2 == np.float32(v) and i2 == i and -(1 << 63) <= k < (1 << 63)
+    best = max(range(len(keys)), key=lambda j: keys[j])
+    assert best == 6
+    assert multigpu.pack_key(2.25, 20) > multigpu.pack_key(2.25, 500)        # equal logits: the lower id wins
+    assert multigpu.pack_key(-1.0, 5) < multigpu.pack_key(-0.5, 5) < multigpu.pack_key(0.5, 5)
+
+
+def _reduce_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    # rank r "owns" token ids [100 r, 100 r + 100): its best (logit, id) per row, as shard keys
+    g = np.random.default_rng(rank)
+    vals = g.standard_normal(16).astype(np.float32)
+    vals[3] = 1.5                                    # an exact tie across ranks: rank 0's id is lower
+    ids = 100 * rank + g.integers(0, 100, 16)
+    keys = torch.tensor([multigpu.pack_key(float(v), int(i)) for v, i in zip(vals, ids)], dtype=torch.int64)
+    dist.all_reduce(keys, op=dist.ReduceOp.MAX)
+    out.put((rank, vals.tolist(), ids.tolist(), keys.tolist()))
+    dist.destroy_process_group()
+
+
+def test_max_all_reduce_of_shard_keys_picks_the_global_argmax():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_reduce_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (_, v0, i0, k0), (_, v1, i1, k1) = res
+    assert k0 == k1
+    for j in range(16):
+        v, i = multigpu.unpack_key(k0[j])
+        want = (v0[j], i0[j]) if (v0[j] > v1[j] or (v0[j] == v1[j] and i0[j] < i1[j])) else (v1[j], i1[j])
+        assert (v, i) == (np.float32(want[0]), want[1])
