@@ -97,6 +97,19 @@ def test_draft_many_distinct_continuations_uses_the_exact_multi_pass_path(ngs, s
     assert small_ctx.get_status() == 0
 
 
+def test_draft_many_short_sequences(ngs, small_ctx):
+    g = np.random.default_rng(8)
+    S, cap, V = 700, 256, 512
+    lens = g.integers(0, cap + 1, S).astype(np.int32)
+    hist = np.full((S, cap), -1, np.int32)
+    for s in range(S):
+        hist[s, :lens[s]] = g.integers(0, 6, lens[s]) if s % 2 else g.integers(0, V, lens[s])
+    T = random_table(V, 6, 4)
+    want = oracle.draft_batch(hist, lens, [3, 1], 5, 12, 6, 3, T)
+    assert_draft_equal(run_draft(small_ctx, hist, lens, [3, 1], 5, 12, 6, 3, T), want)
+    assert small_ctx.get_status() == 0
+
+
 def test_draft_reports_bad_inputs_without_trapping(ngs, small_ctx):
     T = random_table(512, 4, 2)
     hist = np.zeros((2, 16), np.int32)
