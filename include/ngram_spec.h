@@ -189,6 +189,16 @@ int verify_lmhead_keys(spec_ctx* ctx, const void* d_hidden, int M, int vocab_off
 int spec_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_argmax, float* d_max, void* stream);
 
 /*
+ * Ablation counters (Section 5.2: distribution of the accepted length, rank of the accepted draft
+ * among the rows, rows allocated to each strategy).  Adds one decode step's outcome to running
+ * histograms: d_stats = int64 [w+1] accepted length | [B] index of the accepted row (when a > 0) |
+ * [5] strategy of that row (index q, 0 = model) | [5] rows allocated per strategy.  The caller
+ * zeroes d_stats once; d_src is the [S, B] strategy tag from draft_context_ngrams.
+ */
+int spec_accumulate_stats(spec_ctx* ctx, const int32_t* d_acc_len, const int32_t* d_best_row, const int32_t* d_src, int S,
+                          int B, int w, long long* d_stats, void* stream);
+
+/*
  * Test aid: the same tensor-core main loop as the two head calls with a plain store epilogue.
  * d_logits[i, y] = <rows[i, :], unembed[y, :]> for i < m, as float32 [m, V].
  */

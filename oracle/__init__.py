@@ -197,6 +197,18 @@ def accept_commit(drafts, n_drafts, P, hist, lens):
     return acc, best, com
 
 
+def accumulate_stats(acc_len, best_row, src, w: int, stats=None) -> np.ndarray:
+    """Section 5.2 ablation counters: ``[w+1]`` accepted lengths, ``[B]`` accepted row index, ``[5]`` strategy of
+    the accepted row, ``[5]`` rows allocated per strategy (index = q, 0 = model); int64, accumulated."""
+    acc_len, best_row, src = _i32(acc_len), _i32(best_row), _i32(src)
+    S, B = src.shape
+    if stats is None:
+        stats = np.zeros((w + 1) + B + 10, dtype=np.int64)
+    lib().oracle_accumulate_stats(_p(acc_len, C.c_int32), _p(best_row, C.c_int32), _p(src, C.c_int32), S, B, int(w),
+                                  _p(stats, C.c_longlong))
+    return stats
+
+
 # ----------------------------------------------------------------------------- toy-model decode loops
 def toy_greedy(x0: int, n: int, Hall, W) -> list[int]:
     """Plain greedy decoding: x_{t+1} = argmax_y <Hall[x_t], W[y]>, one token per call."""

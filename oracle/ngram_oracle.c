@@ -368,3 +368,32 @@ void oracle_accept_commit(const int32_t* drafts, const int32_t* n_drafts, const 
         best_row[s] = best_b;
     }
 }
+
+/* ------------------------------------------------------------------ ablation counters (Section 5.2)
+ *
+ * Running histograms over decode steps, as in the paper's ablation: accepted length (0..w), row index
+ * of the accepted draft among the B rows (counted when something was accepted), strategy of that row
+ * (q, 0 = model), and rows allocated per strategy.  stats layout: [w+1] [B] [5] [5] int64.
+ */
+void oracle_accumulate_stats(const int32_t* acc_len, const int32_t* best_row, const int32_t* src, int S, int B, int w,
+                             long long* stats) {
+    long long* h_acc = stats;
+    long long* h_row = stats + (w + 1);
+    long long* h_src = h_row + B;
+    long long* h_alloc = h_src + 5;
+    for (int s = 0; s < S; ++s) {
+        for (int b = 0; b < B; ++b) {
+            int q = src[(long)s * B + b];
+            if (q >= 0 && q <= 4) h_alloc[q] += 1;
+        }
+        int a = acc_len[s];
+        if (a < 0) continue; /* the sequence could not commit */
+        h_acc[a > w ? w : a] += 1;
+        if (a > 0) {
+            int b = best_row[s];
+            h_row[b] += 1;
+            int q = src[(long)s * B + b];
+            if (q >= 0 && q <= 4) h_src[q] += 1;
+        }
+    }
+}

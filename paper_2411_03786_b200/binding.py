@@ -60,6 +60,7 @@ def load_library(build: bool = True) -> C.CDLL:
                                          i32p, i32p, vp]
     lib.verify_lmhead_keys.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp]
     lib.spec_unpack_keys.argtypes = [vp, C.c_int, C.c_int, i32p, fp, vp]
+    lib.spec_accumulate_stats.argtypes = [vp, i32p, i32p, i32p, C.c_int, C.c_int, C.c_int, vp, vp]
     lib.spec_debug_logits.argtypes = [vp, vp, C.c_int, fp, vp]
     lib.verify_lmhead_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, i32p, fp, C.c_int, vp]
     lib.spec_launch_count.argtypes = [vp]
@@ -211,6 +212,16 @@ class SpecContext:
         self._check(self._lib.verify_lmhead_keys(self._h, _ptr(hidden, torch.bfloat16), M, int(vocab_offset),
                                                  _ptr(keys, torch.int64), _stream()), "verify_lmhead_keys")
         return keys
+
+    def accumulate_stats(self, acc_len, best_row, src, w: int, stats: torch.Tensor | None = None):
+        """Adds one step to the ablation histograms ([w+1] | [B] | [5] | [5] int64)."""
+        S, B = int(src.shape[0]), int(src.shape[1])
+        if stats is None:
+            stats = torch.zeros((w + 1) + B + 10, dtype=torch.int64, device=src.device)
+        self._check(self._lib.spec_accumulate_stats(self._h, _ptr(acc_len, torch.int32), _ptr(best_row, torch.int32),
+                                                    _ptr(src, torch.int32), S, B, w, _ptr(stats, torch.int64), _stream()),
+                    "spec_accumulate_stats")
+        return stats
 
     def debug_logits(self, rows: torch.Tensor) -> torch.Tensor:
         m = int(rows.shape[0])

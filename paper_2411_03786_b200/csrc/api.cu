@@ -280,6 +280,16 @@ int spec_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_arg
     return launch_unpack_keys(d_keys, M, V_total, d_argmax, d_max, (cudaStream_t)stream);
 }
 
+int spec_accumulate_stats(spec_ctx* ctx, const int32_t* d_acc_len, const int32_t* d_best_row, const int32_t* d_src, int S,
+                          int B, int w, long long* d_stats, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_accumulate_stats: ctx is NULL");
+    if (!d_acc_len || !d_best_row || !d_src || !d_stats) return fail(ctx, SPEC_ERR_ARG, "spec_accumulate_stats: NULL pointer");
+    if (S < 0 || B < 1 || B > kMaxB || w < 1 || w > kMaxW) return fail(ctx, SPEC_ERR_ARG, "spec_accumulate_stats: bad sizes");
+    if (S == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    return launch_stats(ctx, d_acc_len, d_best_row, d_src, S, B, w, d_stats, (cudaStream_t)stream);
+}
+
 int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, void* stream) {
     if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_debug_logits: ctx is NULL");
     if (!d_rows || !d_logits || m < 0) return fail(ctx, SPEC_ERR_ARG, "spec_debug_logits: bad argument");

@@ -223,3 +223,16 @@ def test_fused_verify_accept_equals_the_two_calls_and_the_oracle(ngs, S, B, w):
     assert np.array_equal(l2.cpu().numpy(), l_ref)
     ctx.get_status()
     ctx.close()
+
+
+def test_ablation_counters_match_oracle(ngs, small_ctx):
+    g = np.random.default_rng(12)
+    S, B, w = 500, 10, 6
+    src = g.integers(-1, 5, (S, B)).astype(np.int32)
+    acc = g.integers(-1, w + 1, S).astype(np.int32)
+    best = np.where(acc >= 0, g.integers(0, B, S), -1).astype(np.int32)
+    want = oracle.accumulate_stats(acc, best, src, w)
+    want = oracle.accumulate_stats(acc, best, src, w, stats=want)
+    st = small_ctx.accumulate_stats(dev_i32(acc), dev_i32(best), dev_i32(src), w)
+    st = small_ctx.accumulate_stats(dev_i32(acc), dev_i32(best), dev_i32(src), w, stats=st)
+    assert np.array_equal(st.cpu().numpy(), want)

@@ -188,3 +188,17 @@ def test_rows_reserved_for_the_model_cap_the_context_rows():
     assert d[0].tolist() == [[1, 1], [2, 1], [1, 2], [2, 0]]
     d, nd, src, _ = oracle.draft_batch(hist, lens, [1], 4, 4, 2, 3 | oracle.flag_reserve(9), T)
     assert src[0, :nd[0]].tolist() == [0] * int(nd[0])                        # everything reserved: model rows only
+
+
+def test_ablation_counters_hand_example():
+    # three sequences, B = 3, w = 2
+    src = np.array([[1, 1, 0], [2, 0, -1], [0, 0, 0]], np.int32)
+    acc = np.array([2, 0, -1], np.int32)          # accepted two tokens / nothing / could not commit
+    best = np.array([1, 0, -1], np.int32)
+    st = oracle.accumulate_stats(acc, best, src, w=2)
+    assert st[:3].tolist() == [1, 0, 1]           # accepted lengths 0, 1, 2
+    assert st[3:6].tolist() == [0, 1, 0]          # the accepted row was row 1
+    assert st[6:11].tolist() == [0, 1, 0, 0, 0]   # ... which came from the q = 1 context strategy
+    assert st[11:16].tolist() == [5, 2, 1, 0, 0]  # rows allocated: model 5, q=1 2, q=2 1
+    st2 = oracle.accumulate_stats(acc, best, src, w=2, stats=st.copy())
+    assert np.array_equal(st2, 2 * st)
