@@ -65,7 +65,6 @@ struct GemmParams {
     int a_bytes;      // shared-memory bytes reserved for the A tile of a stage (multiple of 1024)
     int stage_bytes;  // a_bytes + boxes per tile * box bytes
     int stages;       // depth of the operand ring
-    int w_once;       // 1: every row of W is read exactly once (one m-group): hint L2 to evict it first
     int dual;         // 1: A has two m-tiles and every CTA computes both against its W slice (argmax only)
     unsigned long long* keys;
     unsigned int* ticket;
@@ -129,19 +128,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
         : "memory");
-}
-
-// Same with an L2 eviction-priority hint (for data that is streamed once).
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar), "l"(policy)
-        : "memory");
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
 }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
@@ -324,17 +310,13 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2 * (dual ? 2u : 1u);
             // W is a constant of the model: fill the ring with its tiles before waiting for the kernel
             // that produces the activations, then add the A tiles of those stages.
-            const uint64_t w_policy = l2_policy_evict_first();
-            const bool w_once = p.w_once != 0;
             int n_pref = 0;
             for (KbCursor pre(p, MAX_BOXES); n_pref < STAGES && pre.valid; pre.advance(p, MAX_BOXES), ++n_pref) {
                 const uint32_t full = bar_full + 8 * n_pref;
                 const uint32_t sa = tiles + n_pref * STAGE_BYTES;
                 mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_BYTES));
-                for (int j = 0; j < pre.nb; ++j) {
-                    if (w_once) tma_load_2d_hint(sa + A_BYTES + j * BOX_BYTES, &tmB, pre.kb * BLOCK_K, (pre.b0 + j) * BOX_N, full, w_policy);
-                    else tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, pre.kb * BLOCK_K, (pre.b0 + j) * BOX_N, full);
-                }
+                for (int j = 0; j < pre.nb; ++j)
+                    tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, pre.kb * BLOCK_K, (pre.b0 + j) * BOX_N, full);
             }
             grid_dependency_wait();
             for (KbCursor cur(p, MAX_BOXES); cur.valid; cur.advance(p, MAX_BOXES)) {
@@ -346,10 +328,8 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         break;
                     }
                     mbar_expect_tx(full, a_box_bytes + (uint32_t)(cur.nb * BOX_BYTES));
-                    for (int j = 0; j < cur.nb; ++j) {
-                        if (w_once) tma_load_2d_hint(sa + A_BYTES + j * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + j) * BOX_N, full, w_policy);
-                        else tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + j) * BOX_N, full);
-                    }
+                    for (int j = 0; j < cur.nb; ++j)
+                        tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + j) * BOX_N, full);
                 }
                 tma_load_2d(sa, &tmA, cur.kb * BLOCK_K, cur.un.m_tile * BLOCK_M, full);
                 if (dual) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * BLOCK_K, BLOCK_M, full);  // second m-tile
@@ -780,7 +760,6 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.num_kb = (ctx->d + BLOCK_K - 1) / BLOCK_K;
     p.n_mtiles = sh.dual ? 1 : (a_rows + BLOCK_M - 1) / BLOCK_M;  // dual: one unit covers both m-tiles
     p.dual = sh.dual;
-    p.w_once = (sh.dual || p.n_mtiles == 1) ? 1 : 0;
     p.box_n = sh.box_n;
     p.n_boxes = (ctx->V + sh.box_n - 1) / sh.box_n;
     p.n_chunks = sh.n_chunks;
