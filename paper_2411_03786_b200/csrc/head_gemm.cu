@@ -301,7 +301,9 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // The whole warp walks the k-blocks in step; lane j issues W box j and lanes 30 / 31 the A tiles,
+        // so the copies of a stage are issued side by side instead of one after the other.
+        {
             int stage = 0;
             uint32_t phase = 0;
             long long issued = 0;
@@ -314,32 +316,35 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (KbCursor pre(p, MAX_BOXES); n_pref < STAGES && pre.valid; pre.advance(p, MAX_BOXES), ++n_pref) {
                 const uint32_t full = bar_full + 8 * n_pref;
                 const uint32_t sa = tiles + n_pref * STAGE_BYTES;
-                mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_BYTES));
-                for (int j = 0; j < pre.nb; ++j)
-                    tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, pre.kb * BLOCK_K, (pre.b0 + j) * BOX_N, full);
+                if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_BYTES));
+                __syncwarp();
+                if (lane < pre.nb)
+                    tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, pre.kb * BLOCK_K, (pre.b0 + lane) * BOX_N, full);
             }
             grid_dependency_wait();
             for (KbCursor cur(p, MAX_BOXES); cur.valid; cur.advance(p, MAX_BOXES)) {
                 const uint32_t full = bar_full + 8 * stage;
                 const uint32_t sa = tiles + stage * STAGE_BYTES;
                 if (issued >= n_pref) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) {
+                    const bool got = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, got)) {
                         ok = false;
                         break;
                     }
-                    mbar_expect_tx(full, a_box_bytes + (uint32_t)(cur.nb * BOX_BYTES));
-                    for (int j = 0; j < cur.nb; ++j)
-                        tma_load_2d(sa + A_BYTES + j * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + j) * BOX_N, full);
+                    if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(cur.nb * BOX_BYTES));
+                    __syncwarp();
+                    if (lane < cur.nb)
+                        tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + lane) * BOX_N, full);
                 }
-                tma_load_2d(sa, &tmA, cur.kb * BLOCK_K, cur.un.m_tile * BLOCK_M, full);
-                if (dual) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * BLOCK_K, BLOCK_M, full);  // second m-tile
+                if (lane == 31) tma_load_2d(sa, &tmA, cur.kb * BLOCK_K, cur.un.m_tile * BLOCK_M, full);
+                if (dual && lane == 30) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * BLOCK_K, BLOCK_M, full);  // second m-tile
                 ++issued;
                 if (++stage == STAGES) {
                     stage = 0;
                     phase ^= 1u;
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 // Aborting: give copies already in flight a bounded chance to land before the CTA exits.
                 const int pending = issued < STAGES ? (int)issued : STAGES;
                 for (int i = 1; i <= pending; ++i) {
