@@ -505,7 +505,7 @@ def main():
 
 # DRAM bytes per verify launch from the ncu captures summarised under profiles/ (None = not captured
 # for the current kernel).
-TRAFFIC = {"C2": 266.4e6, "C3": 1.676e9}
+TRAFFIC = {"C2": 266.7e6, "C3": 1.668e9}
 
 
 def run_reference(args, c, cfg):
