@@ -160,6 +160,47 @@ def verify(H, W, rows=None):
     return am, mx, gap
 
 
+def e4m3_decode(codes) -> np.ndarray:
+    """Value of each OCP E4M3 code (fp64; 0x7F and 0xFF are NaN)."""
+    lib().oracle_e4m3_decode.restype = C.c_double
+    lib().oracle_e4m3_decode.argtypes = [C.c_uint8]
+    codes = np.asarray(codes, dtype=np.uint8)
+    return np.array([lib().oracle_e4m3_decode(int(c)) for c in codes.reshape(-1)], dtype=np.float64).reshape(codes.shape)
+
+
+def e4m3_encode(values) -> np.ndarray:
+    """Nearest E4M3 code of each fp32 value (ties to even, saturating at 448, zero stored as +0)."""
+    lib().oracle_e4m3_encode.restype = C.c_uint8
+    lib().oracle_e4m3_encode.argtypes = [C.c_float]
+    values = np.asarray(values, dtype=np.float32)
+    return np.array([lib().oracle_e4m3_encode(float(v)) for v in values.reshape(-1)], dtype=np.uint8).reshape(values.shape)
+
+
+def quantize_rows_e4m3(X):
+    """Per-row 8-bit quantisation of a bf16 matrix: ``(codes[R, d] uint8, scale[R] float32)``."""
+    X = _u16(X)
+    R, d = X.shape
+    codes = np.empty((R, d), dtype=np.uint8)
+    scale = np.empty(R, dtype=np.float32)
+    lib().oracle_quantize_rows_e4m3(_p(X, C.c_uint16), C.c_long(R), d, _p(codes, C.c_uint8), _p(scale, C.c_float))
+    return codes, scale
+
+
+def verify_q8(Hq, hscale, Wq, wscale, rows=None):
+    """Greedy next token over the quantised head: ``(argmax[n], max[n], top-2 gap[n])``."""
+    Hq, Wq = np.ascontiguousarray(Hq, dtype=np.uint8), np.ascontiguousarray(Wq, dtype=np.uint8)
+    hscale = np.ascontiguousarray(hscale, dtype=np.float32)
+    wscale = np.ascontiguousarray(wscale, dtype=np.float32)
+    V, d = Wq.shape
+    r, n = _rowsel(rows, Hq.shape[0])
+    am = np.empty(n, dtype=np.int32)
+    mx = np.empty(n, dtype=np.float64)
+    gap = np.empty(n, dtype=np.float64)
+    lib().oracle_verify_rows_q8(_p(Hq, C.c_uint8), _p(hscale, C.c_float), _p(r, C.c_int64), n, _p(Wq, C.c_uint8),
+                                _p(wscale, C.c_float), V, d, _p(am, C.c_int32), _p(mx, C.c_double), _p(gap, C.c_double))
+    return am, mx, gap
+
+
 def unigram_dist2(W, E, rows=None) -> np.ndarray:
     """Section 4.1 "Unigram": squared distance of each output embedding from the mean, in the metric
     induced by the input embeddings (centred rows rounded to bf16, the rest fp64)."""

@@ -11,7 +11,8 @@
  * Pins (tests/test_oracle_*.py): brute force on tiny inputs, a hand-worked
  * example, closed forms (tied unit-norm weights, permutation weights),
  * library matmul/unique cross-checks and the toy-model losslessness
- * invariant.  No routine here is "parity unpinned".
+ * invariant; for the 8-bit head the format's closed form, a nearest-value
+ * search and a library cast.  No routine here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -270,6 +271,97 @@ void oracle_verify_rows(const uint16_t* H, const int64_t* rowsel, int n_rows, co
         long m = rowsel ? (long)rowsel[r] : r;
         double* z = (double*)malloc(sizeof(double) * (size_t)V);
         logits_row(H + m * d, W, V, d, z);
+        int best = 0;
+        for (int y = 1; y < V; ++y)
+            if (z[y] > z[best]) best = y;
+        double second = -INFINITY;
+        for (int y = 0; y < V; ++y)
+            if (y != best && z[y] > second) second = z[y];
+        argmax[r] = best;
+        if (maxval) maxval[r] = z[best];
+        if (gap) gap[r] = z[best] - second;
+        free(z);
+    }
+}
+
+/* ------------------------------------------------------------------ 8-bit head (an addition: the paper only
+ * remarks, in its conclusion, that N-gram speculation composes with quantisation)
+ *
+ * Storage format: OCP 8-bit floating point E4M3 ("FN" variant): 1 sign bit, 4 exponent bits with
+ * bias 7, 3 mantissa bits; no infinities, S.1111.111 is NaN, so the largest finite value is
+ * S.1111.110 = 2^8 * 1.75 = 448; exponent field 0 holds the subnormals m/8 * 2^-6.
+ *
+ * Quantisation of one row x[0..d) of bf16 values (all arithmetic binary32, round to nearest even):
+ *   amax  = max_t |x[t]|                       (exact)
+ *   scale = amax / 448      (1 when amax = 0)  (one division)
+ *   code[t] = E4M3 nearest to x[t] / scale     (one division; ties to the even code; magnitudes
+ *                                               above 448 saturate to 448; a zero result is stored
+ *                                               as +0 whatever its sign)
+ * The head then is z[m][y] = hscale[m] * wscale[y] * sum_t dec(hq[m][t]) * dec(wq[y][t]), fp64 here.
+ */
+double oracle_e4m3_decode(uint8_t c) {
+    int sign = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    double mag;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) mag = ldexp((double)m / 8.0, -6);
+    else mag = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -mag : mag;
+}
+
+/* Nearest E4M3 code of a finite binary32 value.  The 127 finite magnitudes 0x00..0x7E are in
+ * ascending order, so bisect for the largest one <= |y| and then choose between it and its upper
+ * neighbour by exact comparison with their midpoint (both values and the midpoint are exact doubles). */
+uint8_t oracle_e4m3_encode(float y) {
+    double a = fabs((double)y);
+    int lo = 0, hi = 0x7E;
+    if (a >= 448.0) lo = 0x7E;
+    else {
+        while (hi - lo > 1) { /* invariant: dec(lo) <= a < dec(hi) */
+            int mid = (lo + hi) / 2;
+            if (oracle_e4m3_decode((uint8_t)mid) <= a) lo = mid; else hi = mid;
+        }
+        double below = oracle_e4m3_decode((uint8_t)lo), above = oracle_e4m3_decode((uint8_t)(lo + 1));
+        double midpoint = 0.5 * (below + above);
+        if (a > midpoint || (a == midpoint && (lo & 1))) lo = lo + 1;
+    }
+    if (lo == 0) return 0;
+    return (uint8_t)(lo | (signbit(y) ? 0x80 : 0));
+}
+
+void oracle_quantize_rows_e4m3(const uint16_t* X, long n_rows, int d, uint8_t* codes, float* scale) {
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < n_rows; ++r) {
+        const uint16_t* x = X + r * d;
+        float amax = 0.0f;
+        for (int t = 0; t < d; ++t) {
+            float v = fabsf((float)bf16_to_double(x[t]));
+            if (v > amax) amax = v;
+        }
+        float sc = amax > 0.0f ? amax / 448.0f : 1.0f;
+        scale[r] = sc;
+        for (int t = 0; t < d; ++t) {
+            float v = (float)bf16_to_double(x[t]);
+            codes[r * d + t] = oracle_e4m3_encode(v / sc);
+        }
+    }
+}
+
+/* Verification over the quantised head: as oracle_verify_rows, on codes and scales. */
+void oracle_verify_rows_q8(const uint8_t* Hq, const float* hscale, const int64_t* rowsel, int n_rows, const uint8_t* Wq,
+                           const float* wscale, int V, int d, int32_t* argmax, double* maxval, double* gap) {
+    double dec[256];
+    for (int c = 0; c < 256; ++c) dec[c] = oracle_e4m3_decode((uint8_t)c);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < n_rows; ++r) {
+        long m = rowsel ? (long)rowsel[r] : r;
+        const uint8_t* h = Hq + m * d;
+        double* z = (double*)malloc(sizeof(double) * (size_t)V);
+        for (int y = 0; y < V; ++y) {
+            const uint8_t* wy = Wq + (long)y * d;
+            double acc = 0.0;
+            for (int t = 0; t < d; ++t) acc += dec[h[t]] * dec[wy[t]];
+            z[y] = (double)hscale[m] * (double)wscale[y] * acc;
+        }
         int best = 0;
         for (int y = 1; y < V; ++y)
             if (z[y] > z[best]) best = y;
