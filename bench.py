@@ -224,6 +224,7 @@ def main():
     ap.add_argument("--no-table", action="store_true", help="skip timing the one-off table build")
     ap.add_argument("--scaled", action="store_true", help="also time draft/accept on bandwidth-sized batches")
     ap.add_argument("--fuse", action="store_true", help="use verify_accept_commit (one launch) instead of the two calls")
+    ap.add_argument("--fp8", action="store_true", help="also time the 8-bit (E4M3) verification head; reported beside the bf16 numbers")
     ap.add_argument("--no-graph", action="store_true", help="launch the step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -372,6 +373,29 @@ def main():
     torch.cuda.synchronize()
     verify_alone_ms = v0.elapsed_time(v1) / n_ph
 
+    fp8 = None
+    if args.fp8 and c["d"] % 16 == 0:
+        # quantise the head once, then the same back-to-back timing: each call = quantise H (1 launch) + contraction
+        ctx.quantize_head_fp8()
+        scratch8 = (torch.empty((M, c["d"]), dtype=torch.uint8, device=dev), torch.empty(M, dtype=torch.float32, device=dev))
+        out8 = (torch.empty(M, dtype=torch.int32, device=dev), None)
+        for _ in range(5):
+            ctx.verify_lmhead_argmax_fp8(dH, scratch=scratch8, out=out8)
+        f0, f1 = ev(), ev()
+        f0.record()
+        for _ in range(n_ph):
+            ctx.verify_lmhead_argmax_fp8(dH, scratch=scratch8, out=out8)
+        f1.record()
+        torch.cuda.synchronize()
+        fp8_ms = f0.elapsed_time(f1) / n_ph
+        ctx.verify_lmhead_argmax(dH, out=out_v)
+        torch.cuda.synchronize()
+        bytes8 = 1.0 * c["V"] * c["d"] + 4.0 * c["V"] + 2.0 * M * c["d"] + 2.0 * M * c["d"] + 8.0 * M
+        fp8 = {"ms_per_call": fp8_ms, "launches_per_call": 2, "algorithmic_bytes": bytes8,
+               "achieved_gbs": bytes8 / (fp8_ms / 1e3) / 1e9, "frac_of_copy_peak": bytes8 / (fp8_ms / 1e3) / 1e9 / pk["hbm"],
+               "speedup_vs_bf16_verify": verify_alone_ms / fp8_ms,
+               "argmax_agrees_with_bf16": float((out8[0] == out_v[0]).float().mean().item())}
+
     # ---- end to end through the public API with host buffers
     # Pinned staging blobs: [history | lengths] and [hidden states] in, [accepted lengths | committed tokens] out.
     def carve(blob, specs):
@@ -494,6 +518,8 @@ def main():
                         "ms_per_step": e2e_ms / args.steps},
                 "gpu_launches": int(launches) * world, "launch_mode": "eager" if graph is None else "cuda_graph_replay", "roofline": roof, "table_build": table, "cpu_baseline": cpu,
                 "clocks": clk.summary(), "status_bits": status, "copied_fraction": copied}
+        if fp8:
+            line["fp8_verify"] = fp8
         if scaled:
             line["scaled_streams"] = scaled
         print(json.dumps(line))

@@ -199,6 +199,34 @@ int spec_accumulate_stats(spec_ctx* ctx, const int32_t* d_acc_len, const int32_t
                           int B, int w, long long* d_stats, void* stream);
 
 /*
+ * 8-bit verification head.  (The paper computes in bf16 and only remarks, in its conclusion, that the
+ * method composes with quantisation; this is that combination for the memory-bound regime of
+ * Section 3, where the step time is the time to stream the head once: one-byte weights halve it.)
+ *
+ * Format: OCP FP8 E4M3 (1-4-3 bits, bias 7, no infinities, largest finite value 448), one fp32 scale
+ * per row.  Quantisation of a row x (fp32 arithmetic, round to nearest even): amax = max |x|,
+ * scale = amax / 448 (1 for an all-zero row), code = E4M3 nearest to x / scale (ties to the even
+ * code), a zero result stored as +0.  Logit = hscale[m] * wscale[y] * sum_t hq[m][t] * wq[y][t]; the
+ * products are exact and accumulate in fp32 on the tensor cores (tcgen05 kind::f8f6f4).
+ *
+ *   spec_quantize_rows_fp8   d_rows [n_rows, d] bfloat16 -> d_codes [n_rows, d] uint8, d_scale [n_rows].
+ *   spec_quantize_head_fp8   quantises the context's unembedding into caller-owned d_wq [V, d] and
+ *                            d_wscale [V] and adopts them (borrowed: keep them alive).
+ *   spec_set_head_fp8        adopts a head quantised earlier.
+ *   verify_lmhead_argmax_fp8 quantises d_hidden [M, d] bfloat16 into the caller's scratch d_hq [M, d],
+ *                            d_hscale [M], then d_argmax[m] = argmax_y of the logit above (lowest y on
+ *                            exact ties), d_max[m] (or NULL) = that logit.  Two kernels; allocates nothing.
+ * Needs d % 16 == 0 (SPEC_ERR_UNSUPPORTED otherwise); SPEC_ERR_NOT_BUILT before a head is set.
+ * The result can differ from verify_lmhead_argmax wherever the two largest bf16 logits are closer
+ * than the quantisation error; acceptance stays lossless with respect to the quantised model only.
+ */
+int spec_quantize_rows_fp8(spec_ctx* ctx, const void* d_rows, int n_rows, uint8_t* d_codes, float* d_scale, void* stream);
+int spec_quantize_head_fp8(spec_ctx* ctx, uint8_t* d_wq, float* d_wscale, void* stream);
+int spec_set_head_fp8(spec_ctx* ctx, const uint8_t* d_wq, const float* d_wscale);
+int verify_lmhead_argmax_fp8(spec_ctx* ctx, const void* d_hidden, int M, uint8_t* d_hq, float* d_hscale,
+                             int32_t* d_argmax, float* d_max, void* stream);
+
+/*
  * Test aid: the same tensor-core main loop as the two head calls with a plain store epilogue.
  * d_logits[i, y] = <rows[i, :], unembed[y, :]> for i < m, as float32 [m, V].
  */

@@ -308,19 +308,23 @@ double oracle_e4m3_decode(uint8_t c) {
     return sign ? -mag : mag;
 }
 
-/* Nearest E4M3 code of a finite binary32 value.  The 127 finite magnitudes 0x00..0x7E are in
- * ascending order, so bisect for the largest one <= |y| and then choose between it and its upper
- * neighbour by exact comparison with their midpoint (both values and the midpoint are exact doubles). */
-uint8_t oracle_e4m3_encode(float y) {
+/* Nearest E4M3 code of a finite binary32 value.  The 127 finite magnitudes 0x00..0x7E (mag[], from
+ * the decoder) are in ascending order, so bisect for the largest one <= |y| and then choose between it
+ * and its upper neighbour by exact comparison with their midpoint (all three are exact doubles). */
+static void e4m3_magnitudes(double mag[0x7F]) {
+    for (int c = 0; c < 0x7F; ++c) mag[c] = oracle_e4m3_decode((uint8_t)c);
+}
+
+static uint8_t e4m3_encode_with(const double mag[0x7F], float y) {
     double a = fabs((double)y);
     int lo = 0, hi = 0x7E;
     if (a >= 448.0) lo = 0x7E;
     else {
-        while (hi - lo > 1) { /* invariant: dec(lo) <= a < dec(hi) */
+        while (hi - lo > 1) { /* invariant: mag[lo] <= a < mag[hi] */
             int mid = (lo + hi) / 2;
-            if (oracle_e4m3_decode((uint8_t)mid) <= a) lo = mid; else hi = mid;
+            if (mag[mid] <= a) lo = mid; else hi = mid;
         }
-        double below = oracle_e4m3_decode((uint8_t)lo), above = oracle_e4m3_decode((uint8_t)(lo + 1));
+        double below = mag[lo], above = mag[lo + 1];
         double midpoint = 0.5 * (below + above);
         if (a > midpoint || (a == midpoint && (lo & 1))) lo = lo + 1;
     }
@@ -328,7 +332,15 @@ uint8_t oracle_e4m3_encode(float y) {
     return (uint8_t)(lo | (signbit(y) ? 0x80 : 0));
 }
 
+uint8_t oracle_e4m3_encode(float y) {
+    double mag[0x7F];
+    e4m3_magnitudes(mag);
+    return e4m3_encode_with(mag, y);
+}
+
 void oracle_quantize_rows_e4m3(const uint16_t* X, long n_rows, int d, uint8_t* codes, float* scale) {
+    double mag[0x7F];
+    e4m3_magnitudes(mag);
 #pragma omp parallel for schedule(static)
     for (long r = 0; r < n_rows; ++r) {
         const uint16_t* x = X + r * d;
@@ -341,7 +353,7 @@ void oracle_quantize_rows_e4m3(const uint16_t* X, long n_rows, int d, uint8_t* c
         scale[r] = sc;
         for (int t = 0; t < d; ++t) {
             float v = (float)bf16_to_double(x[t]);
-            codes[r * d + t] = oracle_e4m3_encode(v / sc);
+            codes[r * d + t] = e4m3_encode_with(mag, v / sc);
         }
     }
 }

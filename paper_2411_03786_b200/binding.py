@@ -62,6 +62,10 @@ def load_library(build: bool = True) -> C.CDLL:
     lib.spec_unpack_keys.argtypes = [vp, C.c_int, C.c_int, i32p, fp, vp]
     lib.spec_accumulate_stats.argtypes = [vp, i32p, i32p, i32p, C.c_int, C.c_int, C.c_int, vp, vp]
     lib.spec_debug_logits.argtypes = [vp, vp, C.c_int, fp, vp]
+    lib.spec_quantize_rows_fp8.argtypes = [vp, vp, C.c_int, vp, fp, vp]
+    lib.spec_quantize_head_fp8.argtypes = [vp, vp, fp, vp]
+    lib.spec_set_head_fp8.argtypes = [vp, vp, fp]
+    lib.verify_lmhead_argmax_fp8.argtypes = [vp, vp, C.c_int, vp, fp, i32p, fp, vp]
     lib.verify_lmhead_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, i32p, fp, C.c_int, vp]
     lib.spec_launch_count.argtypes = [vp]
     lib.spec_launch_count.restype = C.c_longlong
@@ -222,6 +226,45 @@ class SpecContext:
                                                     _ptr(src, torch.int32), S, B, w, _ptr(stats, torch.int64), _stream()),
                     "spec_accumulate_stats")
         return stats
+
+    def quantize_rows_fp8(self, rows: torch.Tensor, out=None):
+        """Per-row E4M3 quantisation of a bf16 matrix: ``(codes uint8 [n, d], scale float32 [n])``."""
+        n = int(rows.shape[0])
+        if out is None:
+            out = (torch.empty((n, self.d), dtype=torch.uint8, device=rows.device),
+                   torch.empty(n, dtype=torch.float32, device=rows.device))
+        codes, scale = out
+        self._check(self._lib.spec_quantize_rows_fp8(self._h, _ptr(rows, torch.bfloat16), n, _ptr(codes, torch.uint8),
+                                                     _ptr(scale, torch.float32), _stream()), "spec_quantize_rows_fp8")
+        return codes, scale
+
+    def quantize_head_fp8(self):
+        """Builds (and adopts) the 8-bit copy of the unembedding: ``(codes uint8 [V, d], scale float32 [V])``."""
+        dev = self._keep[0].device
+        wq = torch.empty((self.V, self.d), dtype=torch.uint8, device=dev)
+        ws = torch.empty(self.V, dtype=torch.float32, device=dev)
+        self._check(self._lib.spec_quantize_head_fp8(self._h, _ptr(wq), _ptr(ws), _stream()), "spec_quantize_head_fp8")
+        self._keep_fp8 = (wq, ws)
+        return wq, ws
+
+    def set_head_fp8(self, wq: torch.Tensor, ws: torch.Tensor):
+        self._check(self._lib.spec_set_head_fp8(self._h, _ptr(wq, torch.uint8), _ptr(ws, torch.float32)), "spec_set_head_fp8")
+        self._keep_fp8 = (wq, ws)
+
+    def verify_lmhead_argmax_fp8(self, hidden: torch.Tensor, scratch=None, out=None, with_max: bool = False):
+        """``scratch = (codes uint8 [M, d], scale float32 [M])`` receives the quantised hidden states."""
+        M = int(hidden.shape[0])
+        dev = hidden.device
+        if scratch is None:
+            scratch = (torch.empty((M, self.d), dtype=torch.uint8, device=dev), torch.empty(M, dtype=torch.float32, device=dev))
+        if out is None:
+            out = (torch.empty(M, dtype=torch.int32, device=dev),
+                   torch.empty(M, dtype=torch.float32, device=dev) if with_max else None)
+        am, mx = out
+        self._check(self._lib.verify_lmhead_argmax_fp8(self._h, _ptr(hidden, torch.bfloat16), M, _ptr(scratch[0], torch.uint8),
+                                                       _ptr(scratch[1], torch.float32), _ptr(am), _ptr(mx), _stream()),
+                    "verify_lmhead_argmax_fp8")
+        return am, mx
 
     def debug_logits(self, rows: torch.Tensor) -> torch.Tensor:
         m = int(rows.shape[0])

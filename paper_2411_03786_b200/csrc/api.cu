@@ -28,12 +28,13 @@ int check_cuda(spec_ctx* ctx, cudaError_t e, const char* what) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows) {
+int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int elem_bytes) {
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * (cuuint64_t)elem_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows};  // one 128-byte swizzle row wide
     cuuint32_t estr[2] = {1u, 1u};
-    CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+    CUresult r = ctx->encode(tm, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                             const_cast<void*>(base), dims, strides, box,
                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(ctx, SPEC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
@@ -288,6 +289,48 @@ int spec_accumulate_stats(spec_ctx* ctx, const int32_t* d_acc_len, const int32_t
     if (S == 0) return SPEC_OK;
     cudaSetDevice(ctx->device);
     return launch_stats(ctx, d_acc_len, d_best_row, d_src, S, B, w, d_stats, (cudaStream_t)stream);
+}
+
+int spec_quantize_rows_fp8(spec_ctx* ctx, const void* d_rows, int n_rows, uint8_t* d_codes, float* d_scale, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_quantize_rows_fp8: ctx is NULL");
+    if (!d_rows || !d_codes || !d_scale || n_rows < 0) return fail(ctx, SPEC_ERR_ARG, "spec_quantize_rows_fp8: bad argument");
+    if (!aligned16(d_rows) || !aligned16(d_codes)) return fail(ctx, SPEC_ERR_ARG, "spec_quantize_rows_fp8: matrices must be 16-byte aligned");
+    if (ctx->d % 16 != 0) return fail(ctx, SPEC_ERR_UNSUPPORTED, "spec_quantize_rows_fp8: the 8-bit head needs d %% 16 == 0");
+    if (n_rows == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    return launch_quantize_rows(ctx, d_rows, n_rows, d_codes, d_scale, (cudaStream_t)stream);
+}
+
+int spec_quantize_head_fp8(spec_ctx* ctx, uint8_t* d_wq, float* d_wscale, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_quantize_head_fp8: ctx is NULL");
+    int rc = spec_quantize_rows_fp8(ctx, ctx->unembed, ctx->V, d_wq, d_wscale, stream);
+    if (rc) return rc;
+    return spec_set_head_fp8(ctx, d_wq, d_wscale);
+}
+
+int spec_set_head_fp8(spec_ctx* ctx, const uint8_t* d_wq, const float* d_wscale) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_set_head_fp8: ctx is NULL");
+    if (!d_wq || !d_wscale || !aligned16(d_wq)) return fail(ctx, SPEC_ERR_ARG, "spec_set_head_fp8: NULL or misaligned pointer");
+    if (ctx->d % 16 != 0) return fail(ctx, SPEC_ERR_UNSUPPORTED, "spec_set_head_fp8: the 8-bit head needs d %% 16 == 0");
+    ctx->wq = d_wq;
+    ctx->wscale = d_wscale;
+    for (bool& r : ctx->tm_q_ready) r = false;
+    return SPEC_OK;
+}
+
+int verify_lmhead_argmax_fp8(spec_ctx* ctx, const void* d_hidden, int M, uint8_t* d_hq, float* d_hscale, int32_t* d_argmax,
+                             float* d_max, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: ctx is NULL");
+    if (!d_hidden || !d_hq || !d_hscale || !d_argmax) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: NULL pointer");
+    if (!aligned16(d_hidden) || !aligned16(d_hq))
+        return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: d_hidden and d_hq must be 16-byte aligned");
+    if (M < 0 || M > SPEC_MAX_VERIFY_ROWS) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: need 0 <= M <= %d", SPEC_MAX_VERIFY_ROWS);
+    if (!ctx->wq) return fail(ctx, SPEC_ERR_NOT_BUILT, "verify_lmhead_argmax_fp8: call spec_quantize_head_fp8 (or spec_set_head_fp8) first");
+    if (M == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    int rc = launch_quantize_rows(ctx, d_hidden, M, d_hq, d_hscale, (cudaStream_t)stream);
+    if (rc) return rc;
+    return launch_verify_fp8(ctx, d_hq, d_hscale, M, d_argmax, d_max, (cudaStream_t)stream);
 }
 
 int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, void* stream) {

@@ -51,6 +51,11 @@ struct spec_ctx {
     bool tm_w_ready[5] = {false, false, false, false, false};
     CUtensorMap tm_e[5];  // same for the embedding (B operand of the unigram contraction)
     bool tm_e_ready[5] = {false, false, false, false, false};
+    // 8-bit copy of the unembedding (E4M3 codes + one fp32 scale per row), borrowed from the caller
+    const uint8_t* wq = nullptr;
+    const float* wscale = nullptr;
+    CUtensorMap tm_q[5];
+    bool tm_q_ready[5] = {false, false, false, false, false};
     void* d_centred = nullptr;  // unigram scratch: bf16 [V, d] output embeddings minus their mean
     float* d_colsum = nullptr;  // unigram scratch: [64 + 1, d] partial column sums and the mean
     long long launches = 0;
@@ -111,13 +116,17 @@ int fail(spec_ctx* ctx, int code, const char* fmt, ...);
 int check_cuda(spec_ctx* ctx, cudaError_t e, const char* what);
 bool aligned16(const void* p);
 
-// 2-D bf16 row-major [rows, cols] tensor map, 128-byte swizzle, box = [box_rows, 64 elements].
-int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows);
+// 2-D row-major [rows, cols] tensor map of bf16 (elem_bytes = 2) or one-byte elements, 128-byte swizzle,
+// box = [box_rows, 128 bytes].
+int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int elem_bytes = 2);
 
 // head_gemm.cu
 struct AcceptArgs;
 int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st,
                   const AcceptArgs* fuse, long long* d_keys_out, int idx_offset);
+int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale, int M, int32_t* d_argmax, float* d_max,
+                      cudaStream_t st);
+int launch_quantize_rows(spec_ctx* ctx, const void* d_rows, int n_rows, uint8_t* d_codes, float* d_scale, cudaStream_t st);
 int launch_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_argmax, float* d_max, cudaStream_t st);
 int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
                  int32_t* d_ext, cudaStream_t st);

@@ -5,9 +5,12 @@
 //   MODE_TOPK    model bigram table: per row the k largest entries           (build_model_ngram_tables)
 //   MODE_STORE   plain fp32 store, for the logits tolerance check            (spec_debug_logits)
 //   MODE_SUMSQ   model unigram: per row the sum of squares over all columns  (build_model_unigram)
+//   MODE_ARGMAX_Q8  verification over the 8-bit (E4M3) copy of the head          (verify_lmhead_argmax_fp8)
 //
 // A is [a_rows, d] and W is [V, d], both bf16 and K-major, so both operands use the same
-// 128-byte-swizzled K-major shared-memory layout.  One CTA owns the accumulator of a
+// 128-byte-swizzled K-major shared-memory layout.  (The 8-bit mode reads one-byte elements: a
+// 128-byte swizzle row then holds 128 of them and one MMA covers K = 32, so every size counted in
+// bytes below is the same for both element types.)  One CTA owns the accumulator of a
 // 128 x (<=256) tile: TMEM lane = row of A, TMEM column = vocabulary entry.  An epilogue thread
 // therefore owns one row of A and walks its columns in ascending vocabulary order, which makes
 // "lowest token id wins ties" a matter of using a strict comparison.
@@ -38,6 +41,7 @@ namespace ngs {
 
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;               // 64 bf16 = one 128-byte swizzle row
+constexpr int BLOCK_K_Q8 = 128;           // 128 one-byte elements = one 128-byte swizzle row
 constexpr int TILE_N = 256;               // up to 256 columns (rows of W) per tile, in boxes of 16..256 rows
 constexpr int MAX_STAGES = 8;
 constexpr int A_TILE_BYTES = BLOCK_M * BLOCK_K * 2;     // 16 KB: what one MMA reads of A
@@ -48,12 +52,12 @@ constexpr int TMEM_COLS = 512;
 constexpr int GEMM_THREADS = 192;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
-enum { MODE_ARGMAX = 0, MODE_TOPK = 1, MODE_STORE = 2, MODE_SUMSQ = 3 };
+enum { MODE_ARGMAX = 0, MODE_TOPK = 1, MODE_STORE = 2, MODE_SUMSQ = 3, MODE_ARGMAX_Q8 = 4 };
 
 struct GemmParams {
     int a_rows;    // rows of A
     int V;         // rows of W
-    int num_kb;    // ceil(d / 64)
+    int num_kb;    // k-blocks of one swizzle row: ceil(d / 64) for bf16, ceil(d / 128) for one-byte elements
     int n_mtiles;  // ceil(a_rows / 128)
     int box_n;     // rows of W per TMA box (16, 32, 64, 128 or 256)
     int n_boxes;   // ceil(V / box_n)
@@ -79,6 +83,8 @@ struct GemmParams {
     AcceptArgs acc;
     long long* keys_out;  // argmax mode, vocabulary shard: export (value, id) keys instead of ids
     int idx_offset;       // first token id of this shard
+    const float* col_scale;  // 8-bit mode: scale of each row of W (= column of the product)
+    const float* row_scale;  // 8-bit mode: scale of each row of A (only the reported maximum needs it)
 };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
@@ -153,6 +159,15 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same for E4M3 inputs (kind::f8f6f4), one K = 32 slice.
+__device__ __forceinline__ void tc_mma_e4m3(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -182,6 +197,11 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr) {
 // Instruction descriptor for kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N given.
 __device__ __forceinline__ uint32_t make_idesc_bf16(int n_cols) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
+}
+
+// Instruction descriptor for kind::f8f6f4: D = fp32, A = B = E4M3 (format code 0), both K-major.
+__device__ __forceinline__ uint32_t make_idesc_e4m3(int n_cols) {
+    return (1u << 4) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
 }
 
 // Order-preserving map of fp32 onto unsigned integers; key 0 lies below every real value.
@@ -275,6 +295,9 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int* is_last = reinterpret_cast<int*>(tmem_slot + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr bool Q8 = MODE == MODE_ARGMAX_Q8;
+    constexpr bool IS_ARGMAX = MODE == MODE_ARGMAX || MODE == MODE_ARGMAX_Q8;
+    constexpr int KB_ELEMS = Q8 ? BLOCK_K_Q8 : BLOCK_K;  // elements of one k-block (the TMA x step)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -308,7 +331,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
-            const bool dual = MODE == MODE_ARGMAX && p.dual;
+            const bool dual = IS_ARGMAX && p.dual;
             const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2 * (dual ? 2u : 1u);
             // W is a constant of the model: fill the ring with its tiles before waiting for the kernel
             // that produces the activations, then add the A tiles of those stages.
@@ -319,7 +342,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_BYTES));
                 __syncwarp();
                 if (lane < pre.nb)
-                    tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, pre.kb * BLOCK_K, (pre.b0 + lane) * BOX_N, full);
+                    tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, pre.kb * KB_ELEMS, (pre.b0 + lane) * BOX_N, full);
             }
             grid_dependency_wait();
             for (KbCursor cur(p, MAX_BOXES); cur.valid; cur.advance(p, MAX_BOXES)) {
@@ -334,10 +357,10 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(cur.nb * BOX_BYTES));
                     __syncwarp();
                     if (lane < cur.nb)
-                        tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, cur.kb * BLOCK_K, (cur.b0 + lane) * BOX_N, full);
+                        tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, cur.kb * KB_ELEMS, (cur.b0 + lane) * BOX_N, full);
                 }
-                if (lane == 31) tma_load_2d(sa, &tmA, cur.kb * BLOCK_K, cur.un.m_tile * BLOCK_M, full);
-                if (dual && lane == 30) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * BLOCK_K, BLOCK_M, full);  // second m-tile
+                if (lane == 31) tma_load_2d(sa, &tmA, cur.kb * KB_ELEMS, cur.un.m_tile * BLOCK_M, full);
+                if (dual && lane == 30) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * KB_ELEMS, BLOCK_M, full);  // second m-tile
                 ++issued;
                 if (++stage == STAGES) {
                     stage = 0;
@@ -372,14 +395,14 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
                     const int nb = min(MAX_BOXES, un.box_end - b0);
                     // dual: the tile takes both accumulator stages (one per m-tile), so tiles do not overlap
-                    const bool dual = MODE == MODE_ARGMAX && p.dual;
+                    const bool dual = IS_ARGMAX && p.dual;
                     const uint32_t as = dual ? 0u : (tile & 1u), aphase = dual ? (tile & 1u) : ((tile >> 1) & 1u);
                     if (!mbar_wait(bar_tempty + 8 * as, aphase ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t idesc = make_idesc_bf16(nb * BOX_N);
+                    const uint32_t idesc = Q8 ? make_idesc_e4m3(nb * BOX_N) : make_idesc_bf16(nb * BOX_N);
                     const uint32_t d_tmem = tmem_base + as * ACC_COLS;
                     for (int kb = 0; kb < p.num_kb; ++kb) {
                         if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) {
@@ -391,13 +414,17 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const uint64_t adesc = make_kmajor_sw128_desc(sa);
                         const uint64_t bdesc = make_kmajor_sw128_desc(sa + A_BYTES);
 #pragma unroll
-                        for (int k = 0; k < BLOCK_K / 16; ++k)  // +32 bytes (2 x 16 B) per K = 16 slice
-                            tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < 4; ++k) {  // four slices of 32 bytes (2 x 16 B) per swizzle row
+                            if (Q8) tc_mma_e4m3(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            else tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
                         if (dual) {  // the same W tile against the second m-tile, into the other accumulator
                             const uint64_t adesc2 = make_kmajor_sw128_desc(sa + A_TILE_BYTES);
 #pragma unroll
-                            for (int k = 0; k < BLOCK_K / 16; ++k)
-                                tc_mma_bf16(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < 4; ++k) {
+                                if (Q8) tc_mma_e4m3(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                                else tc_mma_bf16(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            }
                         }
                         tc_commit(bar_empty + 8 * stage);  // frees the stage once these MMAs have read it
                         if (++stage == STAGES) {
@@ -424,7 +451,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // running reduction of this row over the unit's columns
             float best_v = MODE == MODE_SUMSQ ? 0.0f : -INFINITY;
             int best_i = 0x7FFFFFFF;
-            const bool dual = MODE == MODE_ARGMAX && p.dual;
+            const bool dual = IS_ARGMAX && p.dual;
             float best_v2 = -INFINITY;  // dual: the row of the second m-tile on this lane
             int best_i2 = 0x7FFFFFFF;
             // Sorted list, value descending, statically indexed so it stays in registers.  The k_tab live
@@ -459,6 +486,17 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             const float v = __uint_as_float(r[j]);
+                            if (j < lim && v > best_v) {
+                                best_v = v;
+                                best_i = cbase + j;
+                            }
+                        }
+                    } else if (MODE == MODE_ARGMAX_Q8) {
+                        // lane j fetches the scale of column cbase + j once; the warp passes it round
+                        const float my_scale = lane < lim ? p.col_scale[cbase + lane] : 0.0f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float v = __uint_as_float(r[j]) * __shfl_sync(0xffffffffu, my_scale, j);
                             if (j < lim && v > best_v) {
                                 best_v = v;
                                 best_i = cbase + j;
@@ -511,9 +549,11 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         tmem_wait_ld();
                         const int cbase = col0 + c * 32;
                         const int lim = n_valid - c * 32;
+                        const float my_scale = Q8 && lane < lim ? p.col_scale[cbase + lane] : 1.0f;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const float v = __uint_as_float(r[j]);
+                            float v = __uint_as_float(r[j]);
+                            if (Q8) v *= __shfl_sync(0xffffffffu, my_scale, j);
                             if (j < lim && v > best_v2) {
                                 best_v2 = v;
                                 best_i2 = cbase + j;
@@ -532,7 +572,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 atomicMax(p.keys + row + BLOCK_M, key);
             }
             if (row < p.a_rows) {
-                if (MODE == MODE_ARGMAX) {
+                if (IS_ARGMAX) {
                     const unsigned long long key =
                         ((unsigned long long)orderable_f32(best_v) << 32) | (unsigned long long)(~(uint32_t)best_i);
                     atomicMax(p.keys + row, key);
@@ -549,7 +589,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             }
         }
-        if (MODE == MODE_ARGMAX) {
+        if (IS_ARGMAX) {
             // The CTA that finishes last turns the merged keys into the outputs and re-arms the scratch.
             const int et = threadIdx.x - 64;
             __threadfence();
@@ -573,7 +613,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         continue;
                     }
                     p.argmax[i] = idx;
-                    if (p.maxv) p.maxv[i] = from_orderable_f32((uint32_t)(key >> 32));
+                    if (p.maxv) p.maxv[i] = from_orderable_f32((uint32_t)(key >> 32)) * (Q8 ? p.row_scale[i] : 1.0f);
                 }
                 if (et == 0) *p.ticket = 0u;
                 if (p.fuse_accept) {
@@ -788,6 +828,8 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.acc = AcceptArgs{};
     p.keys_out = nullptr;
     p.idx_offset = 0;
+    p.col_scale = nullptr;
+    p.row_scale = nullptr;
 }
 
 int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st,
@@ -813,6 +855,89 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, tmA, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax launch");
+}
+
+// ------------------------------------------------------------------------------------------ 8-bit head
+// Per-row quantisation of a bf16 matrix to E4M3 (all arithmetic fp32, round to nearest even):
+//   amax = max |x|, scale = amax / 448 (1 for an all-zero row), code = e4m3(x / scale), zero stored as +0.
+// One CTA per row; a thread handles 8 consecutive elements at a time.
+__device__ __forceinline__ uint32_t e4m3_pair(float lo, float hi) {
+    uint16_t r;  // cvt packs {hi, lo}: the first source lands in the upper byte
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    uint32_t v = r;
+    if ((v & 0x007Fu) == 0u) v &= 0xFF00u;  // -0 -> +0
+    if ((v & 0x7F00u) == 0u) v &= 0x00FFu;
+    return v;
+}
+
+__global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const __nv_bfloat16* __restrict__ X, int d,
+                                                                 uint8_t* __restrict__ codes, float* __restrict__ scale) {
+    __shared__ float warp_max[8];
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const size_t row = blockIdx.x;
+    const uint4* x8 = reinterpret_cast<const uint4*>(X + row * d);  // 8 bf16 per load; d % 16 == 0
+    const int n8 = d / 8;
+    float amax = 0.0f;
+    for (int i = threadIdx.x; i < n8; i += blockDim.x) {
+        const uint4 v = x8[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            amax = fmaxf(amax, fabsf(__uint_as_float(w[j] << 16)));
+            amax = fmaxf(amax, fabsf(__uint_as_float(w[j] & 0xFFFF0000u)));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    amax = warp_max[0];
+#pragma unroll
+    for (int j = 1; j < 8; ++j) amax = fmaxf(amax, warp_max[j]);
+    const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+    if (threadIdx.x == 0) scale[row] = sc;
+    uint2* out = reinterpret_cast<uint2*>(codes + row * d);
+    for (int i = threadIdx.x; i < n8; i += blockDim.x) {
+        const uint4 v = x8[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t pair[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            pair[j] = e4m3_pair(__fdiv_rn(__uint_as_float(w[j] << 16), sc), __fdiv_rn(__uint_as_float(w[j] & 0xFFFF0000u), sc));
+        out[i] = make_uint2(pair[0] | (pair[1] << 16), pair[2] | (pair[3] << 16));
+    }
+}
+
+int launch_quantize_rows(spec_ctx* ctx, const void* d_rows, int n_rows, uint8_t* d_codes, float* d_scale, cudaStream_t st) {
+    cudaError_t e = launch_pdl(quantize_rows_e4m3_kernel, dim3(n_rows), dim3(256), 0, st, (const __nv_bfloat16*)d_rows, ctx->d,
+                               d_codes, d_scale);
+    ctx->launches += 1;
+    return check_cuda(ctx, e, "8-bit quantisation launch");
+}
+
+int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale, int M, int32_t* d_argmax, float* d_max,
+                      cudaStream_t st) {
+    int rc = set_smem_attr<MODE_ARGMAX_Q8, 1>(ctx);
+    if (rc) return rc;
+    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
+    if (!ctx->tm_q_ready[sh.box_idx]) {
+        if ((rc = make_tensor_map(ctx, &ctx->tm_q[sh.box_idx], ctx->wq, ctx->V, ctx->d, sh.box_n, 1))) return rc;
+        ctx->tm_q_ready[sh.box_idx] = true;
+    }
+    CUtensorMap tmA;
+    if ((rc = make_tensor_map(ctx, &tmA, d_hq, M, ctx->d, sh.a_box_rows, 1))) return rc;
+    GemmParams p;
+    fill_common(ctx, p, M, sh);
+    p.num_kb = (ctx->d + BLOCK_K_Q8 - 1) / BLOCK_K_Q8;
+    p.argmax = d_argmax;
+    p.maxv = d_max;
+    p.col_scale = ctx->wscale;
+    p.row_scale = d_hscale;
+    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX_Q8, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, tmA,
+                               ctx->tm_q[sh.box_idx], p);
+    ctx->launches += 1;
+    return check_cuda(ctx, e, "verify_lmhead_argmax_fp8 launch");
 }
 
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st) {
