@@ -216,6 +216,8 @@ int spec_accumulate_stats(spec_ctx* ctx, const int32_t* d_acc_len, const int32_t
  *   verify_lmhead_argmax_fp8 quantises d_hidden [M, d] bfloat16 into the caller's scratch d_hq [M, d],
  *                            d_hscale [M], then d_argmax[m] = argmax_y of the logit above (lowest y on
  *                            exact ties), d_max[m] (or NULL) = that logit.  Two kernels; allocates nothing.
+ *                            d_hidden = NULL: d_hq / d_hscale already hold the quantised hidden states
+ *                            (a model whose last layer emits them in this format); one kernel.
  * Needs d % 16 == 0 (SPEC_ERR_UNSUPPORTED otherwise); SPEC_ERR_NOT_BUILT before a head is set.
  * The result can differ from verify_lmhead_argmax wherever the two largest bf16 logits are closer
  * than the quantisation error; acceptance stays lossless with respect to the quantised model only.

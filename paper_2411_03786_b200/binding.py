@@ -251,10 +251,11 @@ class SpecContext:
         self._check(self._lib.spec_set_head_fp8(self._h, _ptr(wq, torch.uint8), _ptr(ws, torch.float32)), "spec_set_head_fp8")
         self._keep_fp8 = (wq, ws)
 
-    def verify_lmhead_argmax_fp8(self, hidden: torch.Tensor, scratch=None, out=None, with_max: bool = False):
-        """``scratch = (codes uint8 [M, d], scale float32 [M])`` receives the quantised hidden states."""
-        M = int(hidden.shape[0])
-        dev = hidden.device
+    def verify_lmhead_argmax_fp8(self, hidden: torch.Tensor | None, scratch=None, out=None, with_max: bool = False):
+        """``scratch = (codes uint8 [M, d], scale float32 [M])`` receives the quantised hidden states; with
+        ``hidden=None`` it already holds them."""
+        M = int(hidden.shape[0]) if hidden is not None else int(scratch[0].shape[0])
+        dev = hidden.device if hidden is not None else scratch[0].device
         if scratch is None:
             scratch = (torch.empty((M, self.d), dtype=torch.uint8, device=dev), torch.empty(M, dtype=torch.float32, device=dev))
         if out is None:

@@ -41,6 +41,25 @@ int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, 
     return SPEC_OK;
 }
 
+int a_tensor_map(spec_ctx* ctx, const CUtensorMap** out, const void* base, int rows, int cols, int box_rows, int elem_bytes) {
+    for (auto& m : ctx->a_maps)
+        if (m.base == base && m.rows == rows && m.box_rows == box_rows && m.elem_bytes == elem_bytes) {
+            *out = &m.tm;
+            return SPEC_OK;
+        }
+    spec_ctx::AMap& m = ctx->a_maps[ctx->a_map_next];
+    ctx->a_map_next = (ctx->a_map_next + 1) % 4;
+    m.base = nullptr;
+    int rc = make_tensor_map(ctx, &m.tm, base, rows, cols, box_rows, elem_bytes);
+    if (rc) return rc;
+    m.base = base;
+    m.rows = rows;
+    m.box_rows = box_rows;
+    m.elem_bytes = elem_bytes;
+    *out = &m.tm;
+    return SPEC_OK;
+}
+
 __global__ void round_f32_to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, size_t n) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -321,15 +340,17 @@ int spec_set_head_fp8(spec_ctx* ctx, const uint8_t* d_wq, const float* d_wscale)
 int verify_lmhead_argmax_fp8(spec_ctx* ctx, const void* d_hidden, int M, uint8_t* d_hq, float* d_hscale, int32_t* d_argmax,
                              float* d_max, void* stream) {
     if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: ctx is NULL");
-    if (!d_hidden || !d_hq || !d_hscale || !d_argmax) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: NULL pointer");
-    if (!aligned16(d_hidden) || !aligned16(d_hq))
+    if (!d_hq || !d_hscale || !d_argmax) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: NULL pointer");
+    if ((d_hidden && !aligned16(d_hidden)) || !aligned16(d_hq))
         return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: d_hidden and d_hq must be 16-byte aligned");
     if (M < 0 || M > SPEC_MAX_VERIFY_ROWS) return fail(ctx, SPEC_ERR_ARG, "verify_lmhead_argmax_fp8: need 0 <= M <= %d", SPEC_MAX_VERIFY_ROWS);
     if (!ctx->wq) return fail(ctx, SPEC_ERR_NOT_BUILT, "verify_lmhead_argmax_fp8: call spec_quantize_head_fp8 (or spec_set_head_fp8) first");
     if (M == 0) return SPEC_OK;
     cudaSetDevice(ctx->device);
-    int rc = launch_quantize_rows(ctx, d_hidden, M, d_hq, d_hscale, (cudaStream_t)stream);
-    if (rc) return rc;
+    if (d_hidden) {  // NULL: the caller's own producer already left codes and scales in d_hq / d_hscale
+        int rc = launch_quantize_rows(ctx, d_hidden, M, d_hq, d_hscale, (cudaStream_t)stream);
+        if (rc) return rc;
+    }
     return launch_verify_fp8(ctx, d_hq, d_hscale, M, d_argmax, d_max, (cudaStream_t)stream);
 }
 

@@ -56,6 +56,14 @@ struct spec_ctx {
     const float* wscale = nullptr;
     CUtensorMap tm_q[5];
     bool tm_q_ready[5] = {false, false, false, false, false};
+    // tensor maps of the most recent A operands (hidden states), so a decode loop that verifies from the
+    // same buffer every step does not re-encode the map on every call
+    struct AMap {
+        const void* base = nullptr;
+        int rows = 0, box_rows = 0, elem_bytes = 0;
+        CUtensorMap tm;
+    } a_maps[4];
+    int a_map_next = 0;
     void* d_centred = nullptr;  // unigram scratch: bf16 [V, d] output embeddings minus their mean
     float* d_colsum = nullptr;  // unigram scratch: [64 + 1, d] partial column sums and the mean
     long long launches = 0;
@@ -119,6 +127,9 @@ bool aligned16(const void* p);
 // 2-D row-major [rows, cols] tensor map of bf16 (elem_bytes = 2) or one-byte elements, 128-byte swizzle,
 // box = [box_rows, 128 bytes].
 int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int elem_bytes = 2);
+
+// Cached form of make_tensor_map for an A operand; *out stays valid until four other operands were mapped.
+int a_tensor_map(spec_ctx* ctx, const CUtensorMap** out, const void* base, int rows, int cols, int box_rows, int elem_bytes = 2);
 
 // head_gemm.cu
 struct AcceptArgs;

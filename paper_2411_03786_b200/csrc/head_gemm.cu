@@ -839,8 +839,8 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
     const CUtensorMap* tmW;
     if ((rc = w_map(ctx, sh, &tmW))) return rc;
-    CUtensorMap tmA;
-    if ((rc = make_tensor_map(ctx, &tmA, d_hidden, M, ctx->d, sh.a_box_rows))) return rc;
+    const CUtensorMap* tmA;
+    if ((rc = a_tensor_map(ctx, &tmA, d_hidden, M, ctx->d, sh.a_box_rows))) return rc;
     GemmParams p;
     fill_common(ctx, p, M, sh);
     p.argmax = d_argmax;
@@ -852,7 +852,7 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     }
     p.keys_out = d_keys_out;
     p.idx_offset = idx_offset;
-    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, tmA, *tmW, p);
+    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax launch");
 }
@@ -925,8 +925,8 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
         if ((rc = make_tensor_map(ctx, &ctx->tm_q[sh.box_idx], ctx->wq, ctx->V, ctx->d, sh.box_n, 1))) return rc;
         ctx->tm_q_ready[sh.box_idx] = true;
     }
-    CUtensorMap tmA;
-    if ((rc = make_tensor_map(ctx, &tmA, d_hq, M, ctx->d, sh.a_box_rows, 1))) return rc;
+    const CUtensorMap* tmA;
+    if ((rc = a_tensor_map(ctx, &tmA, d_hq, M, ctx->d, sh.a_box_rows, 1))) return rc;
     GemmParams p;
     fill_common(ctx, p, M, sh);
     p.num_kb = (ctx->d + BLOCK_K_Q8 - 1) / BLOCK_K_Q8;
@@ -934,7 +934,7 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
     p.maxv = d_max;
     p.col_scale = ctx->wscale;
     p.row_scale = d_hscale;
-    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX_Q8, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, tmA,
+    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX_Q8, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA,
                                ctx->tm_q[sh.box_idx], p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax_fp8 launch");

@@ -62,6 +62,10 @@ def test_fp8_verify_matches_oracle(ngs, V, d, M):
         bad = am != ref_am
         assert not (bad & (gap >= TOL)).any(), f"{bad.sum()} mismatches with clear margins"
         assert np.abs(mx - ref_mx).max() <= TOL
+    # hidden states quantised by the caller beforehand
+    scratch = ctx.quantize_rows_fp8(dev_bf16(H))
+    am2, _ = ctx.verify_lmhead_argmax_fp8(None, scratch=scratch)
+    assert np.array_equal(am2.cpu().numpy(), am)
     assert ctx.get_status() == 0
     ctx.close()
 

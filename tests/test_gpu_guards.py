@@ -14,19 +14,25 @@ SENT = -123456789
 
 def guarded(shape, dtype):
     n = int(np.prod(shape))
-    buf = torch.full((n + 2 * GUARD,), SENT, dtype=dtype, device="cuda")
+    byte = dtype == torch.uint8          # E4M3 codes: sentinel 0xA5, poison 0x7F (the NaN code, never produced)
+    buf = torch.full((n + 2 * GUARD,), 0xA5 if byte else SENT, dtype=dtype, device="cuda")
     view = buf[GUARD:GUARD + n].view(shape)
-    view.fill_(-77)                      # poison: stale values cannot pass for results
+    view.fill_(0x7F if byte else -77)    # poison: stale values cannot pass for results
     return buf, view
 
 
 def intact(buf):
-    return bool((buf[:GUARD] == SENT).all() and (buf[-GUARD:] == SENT).all())
+    sent = 0xA5 if buf.dtype == torch.uint8 else SENT
+    return bool((buf[:GUARD] == sent).all() and (buf[-GUARD:] == sent).all())
+
+
+def unwritten(view):
+    return bool((view == (0x7F if view.dtype == torch.uint8 else -77)).any())
 
 
 def test_outputs_stay_inside_their_buffers_and_repeat():
     import paper_2411_03786_b200 as ngs
-    V, d, k, w, B, S, cap = 1000, 200, 10, 5, 8, 3, 408
+    V, d, k, w, B, S, cap = 1000, 208, 10, 5, 8, 3, 408
     E = synth.gaussian_weights(V, d, 1.0, 1, "E")
     W = synth.gaussian_weights(V, d, 1.0, 1, "W")
     ctx = ngs.SpecContext(dev_bf16(E), dev_bf16(W))
@@ -60,12 +66,18 @@ def test_outputs_stay_inside_their_buffers_and_repeat():
         assert lib.accept_and_commit(h, P(drafts), P(nd), P(am), S, B, w, P(hist), P(lens), cap, P(acc), P(best), P(com), None) == 0
         logits = out("logits", (5, V), torch.float32)
         assert lib.spec_debug_logits(h, P(H), 5, P(logits), None) == 0
+        wq, ws = out("wq", (V, d), torch.uint8), out("ws", (V,), torch.float32)
+        assert lib.spec_quantize_head_fp8(h, P(wq), P(ws), None) == 0
+        hq, hs = out("hq", (M, d), torch.uint8), out("hs", (M,), torch.float32)
+        am8, mx8 = out("am8", (M,)), out("mx8", (M,), torch.float32)
+        assert lib.verify_lmhead_argmax_fp8(h, P(H), M, P(hq), P(hs), P(am8), P(mx8), None) == 0
         torch.cuda.synchronize()
         assert ctx.get_status() == 0
         for name, (buf, view) in bufs.items():
             assert intact(buf), f"{name}: guard region overwritten"
-        for name in ("tab", "val", "ext", "uni", "d2", "nd", "src", "cnt", "am", "mx", "acc", "best", "logits"):
-            assert not (bufs[name][1] == -77).any(), f"{name}: element left unwritten"
+        for name in ("tab", "val", "ext", "uni", "d2", "nd", "src", "cnt", "am", "mx", "acc", "best", "logits", "wq", "ws", "hq", "hs",
+                     "am8", "mx8"):
+            assert not unwritten(bufs[name][1]), f"{name}: element left unwritten"
         results.append({n: v.clone() for n, (b, v) in bufs.items()})
     for name in results[0]:
         assert torch.equal(results[0][name], results[1][name]), f"{name}: two identical calls disagree"
