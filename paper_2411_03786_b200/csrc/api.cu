@@ -41,6 +41,14 @@ int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, 
     return SPEC_OK;
 }
 
+int make_w_maps(spec_ctx* ctx, WMaps* maps, const void* base, int elem_bytes) {
+    for (int i = 0; i < 5; ++i) {
+        int rc = make_tensor_map(ctx, &maps->m[i], base, ctx->V, ctx->d, 256 >> i, elem_bytes);
+        if (rc) return rc;
+    }
+    return SPEC_OK;
+}
+
 int a_tensor_map(spec_ctx* ctx, const CUtensorMap** out, const void* base, int rows, int cols, int box_rows, int elem_bytes) {
     for (auto& m : ctx->a_maps)
         if (m.base == base && m.rows == rows && m.box_rows == box_rows && m.elem_bytes == elem_bytes) {
@@ -135,11 +143,11 @@ int spec_init(spec_ctx** out, const void* d_embed, const void* d_unembed, int dt
         cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st);
         cudaMemsetAsync(ctx->d_keys, 0, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS, st);
         cudaMemsetAsync(ctx->d_ticket, 0, sizeof(unsigned int), st);
-        if ((rc = make_tensor_map(ctx, &ctx->tm_w[1], ctx->unembed, V, d, 32))) {
+        if ((rc = make_w_maps(ctx, &ctx->tm_w, ctx->unembed, 2))) {
             strncpy(g_err, ctx->err, 255);
             break;
         }
-        ctx->tm_w_ready[1] = true;
+        ctx->tm_w_ready = true;
         if ((rc = check_cuda(nullptr, cudaStreamSynchronize(st), "spec_init: stream sync"))) break;
     } while (0);
     if (rc != SPEC_OK) {
@@ -333,7 +341,7 @@ int spec_set_head_fp8(spec_ctx* ctx, const uint8_t* d_wq, const float* d_wscale)
     if (ctx->d % 16 != 0) return fail(ctx, SPEC_ERR_UNSUPPORTED, "spec_set_head_fp8: the 8-bit head needs d %% 16 == 0");
     ctx->wq = d_wq;
     ctx->wscale = d_wscale;
-    for (bool& r : ctx->tm_q_ready) r = false;
+    ctx->tm_q_ready = false;
     return SPEC_OK;
 }
 

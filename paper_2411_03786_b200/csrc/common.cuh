@@ -21,6 +21,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Tensor maps of one [V, d] matrix as the B operand of the head contraction, with 256-, 128-, 64-, 32- and
+// 16-row boxes: a tile of any multiple of 16 rows is fetched with one copy per set bit of its row count.
+struct WMaps {
+    CUtensorMap m[5];
+};
+
 }  // namespace ngs
 
 struct spec_ctx {
@@ -45,17 +51,16 @@ struct spec_ctx {
     const int32_t* ext = nullptr;
     int w_ext = 0;
     ngs::EncodeTiledFn encode = nullptr;
-    // B operand of every contraction: tensor maps of the unembedding with 16/32/64/128/256-row boxes,
-    // encoded on first use (host-side work only)
-    CUtensorMap tm_w[5];
-    bool tm_w_ready[5] = {false, false, false, false, false};
-    CUtensorMap tm_e[5];  // same for the embedding (B operand of the unigram contraction)
-    bool tm_e_ready[5] = {false, false, false, false, false};
+    // B operand of every contraction: tensor maps of the unembedding, encoded on first use (host-side work only)
+    ngs::WMaps tm_w;
+    bool tm_w_ready = false;
+    ngs::WMaps tm_e;  // same for the embedding (B operand of the unigram contraction)
+    bool tm_e_ready = false;
     // 8-bit copy of the unembedding (E4M3 codes + one fp32 scale per row), borrowed from the caller
     const uint8_t* wq = nullptr;
     const float* wscale = nullptr;
-    CUtensorMap tm_q[5];
-    bool tm_q_ready[5] = {false, false, false, false, false};
+    ngs::WMaps tm_q;
+    bool tm_q_ready = false;
     // tensor maps of the most recent A operands (hidden states), so a decode loop that verifies from the
     // same buffer every step does not re-encode the map on every call
     struct AMap {
@@ -128,6 +133,8 @@ bool aligned16(const void* p);
 // box = [box_rows, 128 bytes].
 int make_tensor_map(spec_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int elem_bytes = 2);
 
+// The five maps of a [V, d] B operand (see WMaps).
+int make_w_maps(spec_ctx* ctx, WMaps* maps, const void* base, int elem_bytes);
 // Cached form of make_tensor_map for an A operand; *out stays valid until four other operands were mapped.
 int a_tensor_map(spec_ctx* ctx, const CUtensorMap** out, const void* base, int rows, int cols, int box_rows, int elem_bytes = 2);
 

@@ -10,6 +10,10 @@
 // actual tokens, so grouping is exact.  If a sequence has more distinct continuations than the
 // table holds, the scan is repeated in R passes, pass r keeping only the groups whose hash falls
 // in residue class r, and the per-pass winners are merged: still exact, only slower.
+//
+// A history of up to 8192 tokens is first copied into shared memory (one round of 128-bit loads);
+// the scan, the key comparisons and the candidate rows then never wait for global memory again,
+// which is what the latency of a single short sequence is made of.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -37,6 +41,8 @@ struct DraftParams {
     int* status;
     int slots;       // hash table size (power of two)
     int max_groups;  // slots / 2
+    int stage_hist;  // 1: copy the history into shared memory first (single CTA, short history)
+    int hist_off;    // where that copy lives, in ints from the start of the hash table
 };
 
 constexpr int kMaxPasses = 1024;
@@ -155,6 +161,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     const int s = (int)blockIdx.x / csize;
     const int32_t* __restrict__ h = P.hist + (size_t)s * P.cap;
     const int w = P.w;
+    int32_t* hist_s = rep + P.hist_off;
 
     grid_launch_dependents();  // the verify kernel may start streaming weights while this one runs
     grid_dependency_wait();    // history and lengths come from the previous step's commit
@@ -162,6 +169,15 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     if (L < 0 || L > P.cap) {
         if (tid == 0 && leader) atomicOr(P.status, SPEC_STATUS_CAPACITY);
         L = 0;
+    }
+    if (P.stage_hist) {
+        const int4* g4 = reinterpret_cast<const int4*>(h);
+        int4* s4 = reinterpret_cast<int4*>(hist_s);
+        const int n4 = (L + 3) >> 2;  // cap % 4 == 0 and L <= cap: the last vector stays inside the row
+#pragma unroll 4
+        for (int i = tid; i < n4; i += nthr) s4[i] = g4[i];
+        __syncthreads();
+        h = hist_s;
     }
     if (tid < kMaxQ) sm->tq[tid] = (tid < L) ? h[L - 1 - tid] : -2;
     if (tid < kMaxNQ) sm->n_run[tid] = 0;
@@ -543,7 +559,10 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     while (csize < 8 && (int)(csize * 2) * 16384 <= cap && (long long)S * (csize * 2) <= ctx->num_sms) csize <<= 1;
     const size_t table_bytes = (size_t)slots * 3 * sizeof(int) + (size_t)P.max_groups * sizeof(int);
     const size_t cand_bytes = (size_t)(n_q * topk + kMaxKTab) * w * sizeof(int32_t);  // aliases the table
-    const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + (table_bytes > cand_bytes ? table_bytes : cand_bytes);
+    const size_t work_bytes = ((table_bytes > cand_bytes ? table_bytes : cand_bytes) + 15) & ~size_t(15);
+    P.stage_hist = (csize == 1 && cap <= 8192) ? 1 : 0;
+    P.hist_off = (int)(work_bytes / sizeof(int));
+    const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + work_bytes + (P.stage_hist ? (size_t)cap * sizeof(int32_t) : 0);
     static bool attr_set[64] = {false};
     bool& attr_done = attr_set[ctx->device & 63];
     if (!attr_done) {

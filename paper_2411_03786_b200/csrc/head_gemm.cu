@@ -213,6 +213,32 @@ __device__ __forceinline__ float from_orderable_f32(uint32_t u) {
     return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
 }
 
+// Arg max of 32 consecutive columns as a tree of independent comparisons (depth 5 instead of a chain
+// of 32 dependent ones: this runs at the very end of a memory-bound launch, where nothing hides it).
+// A right-hand (higher) column wins only if strictly larger, so equal values keep the lowest column.
+// Returns the winning value and its offset in [0, 32).
+__device__ __forceinline__ void chunk_argmax(const float (&v)[32], float& best, int& off) {
+    float a16[16];
+    int i16[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const bool hi = v[2 * j + 1] > v[2 * j];
+        a16[j] = hi ? v[2 * j + 1] : v[2 * j];
+        i16[j] = 2 * j + (hi ? 1 : 0);
+    }
+#pragma unroll
+    for (int n = 8; n >= 1; n >>= 1) {
+#pragma unroll
+        for (int j = 0; j < n; ++j) {
+            const bool hi = a16[2 * j + 1] > a16[2 * j];
+            a16[j] = hi ? a16[2 * j + 1] : a16[2 * j];
+            i16[j] = hi ? i16[2 * j + 1] : i16[2 * j];
+        }
+    }
+    best = a16[0];
+    off = i16[0];
+}
+
 // ------------------------------------------------------------------------------------------ work units
 struct Unit {
     int m_tile, chunk, box_begin, box_end;
@@ -275,13 +301,13 @@ struct KbCursor {
 // KT = capacity of the per-thread top-k list (registers); only MODE_TOPK uses it.
 template <int MODE, int KT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ WMaps tmB, const GemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;               // operand stages, 1024-byte aligned
     unsigned char* tiles_ptr = smem_raw + (tiles - raw);
     const int STAGES = p.stages, STAGE_BYTES = p.stage_bytes, A_BYTES = p.a_bytes;
-    const int BOX_N = p.box_n, BOX_BYTES = p.box_n * BLOCK_K * 2, MAX_BOXES = TILE_N / p.box_n;
+    const int BOX_N = p.box_n, MAX_BOXES = TILE_N / p.box_n;
     // The MMA always reads a 128-row A tile; when fewer rows are loaded the rest of that window is
     // whatever follows in shared memory (rows that no output uses), so keep the window in bounds.
     uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES + (A_TILE_BYTES - A_BYTES));
@@ -299,6 +325,8 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr bool IS_ARGMAX = MODE == MODE_ARGMAX || MODE == MODE_ARGMAX_Q8;
     constexpr int KB_ELEMS = Q8 ? BLOCK_K_Q8 : BLOCK_K;  // elements of one k-block (the TMA x step)
 
+    if (warp == 0 && lane < 6)  // the descriptors' first use would otherwise pay their fetch on the critical path
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(lane < 5 ? &tmB.m[lane] : &tmA)) : "memory");
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -324,8 +352,9 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        // The whole warp walks the k-blocks in step; lane j issues W box j and lanes 30 / 31 the A tiles,
-        // so the copies of a stage are issued side by side instead of one after the other.
+        // The whole warp walks the k-blocks in step; lanes 0..4 issue the W tile as one copy per set bit of
+        // its row count (256, 128, 64, 32, 16 rows) and lanes 30 / 31 the A tiles, so the copies of a stage
+        // are issued side by side instead of one after the other.
         {
             int stage = 0;
             uint32_t phase = 0;
@@ -333,16 +362,24 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             bool ok = true;
             const bool dual = IS_ARGMAX && p.dual;
             const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2 * (dual ? 2u : 1u);
+            const int my_rows = 256 >> lane;  // lanes 0..4: the piece size this lane copies
+            // piece of `rows` (a multiple of 16, at most 256) for this lane: the rows above it come first
+            auto w_piece = [&](uint32_t sa, int kb, int b0, int nb, uint32_t full) {
+                const int rows = nb * BOX_N;
+                if (lane < 5 && (rows & my_rows)) {
+                    const int before = rows & ~(2 * my_rows - 1);
+                    tma_load_2d(sa + A_BYTES + before * 128, &tmB.m[lane], kb * KB_ELEMS, b0 * BOX_N + before, full);
+                }
+            };
             // W is a constant of the model: fill the ring with its tiles before waiting for the kernel
             // that produces the activations, then add the A tiles of those stages.
             int n_pref = 0;
             for (KbCursor pre(p, MAX_BOXES); n_pref < STAGES && pre.valid; pre.advance(p, MAX_BOXES), ++n_pref) {
                 const uint32_t full = bar_full + 8 * n_pref;
                 const uint32_t sa = tiles + n_pref * STAGE_BYTES;
-                if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_BYTES));
+                if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_N * 128));
                 __syncwarp();
-                if (lane < pre.nb)
-                    tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, pre.kb * KB_ELEMS, (pre.b0 + lane) * BOX_N, full);
+                w_piece(sa, pre.kb, pre.b0, pre.nb, full);
             }
             grid_dependency_wait();
             for (KbCursor cur(p, MAX_BOXES); cur.valid; cur.advance(p, MAX_BOXES)) {
@@ -354,10 +391,9 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         ok = false;
                         break;
                     }
-                    if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(cur.nb * BOX_BYTES));
+                    if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(cur.nb * BOX_N * 128));
                     __syncwarp();
-                    if (lane < cur.nb)
-                        tma_load_2d(sa + A_BYTES + lane * BOX_BYTES, &tmB, cur.kb * KB_ELEMS, (cur.b0 + lane) * BOX_N, full);
+                    w_piece(sa, cur.kb, cur.b0, cur.nb, full);
                 }
                 if (lane == 31) tma_load_2d(sa, &tmA, cur.kb * KB_ELEMS, cur.un.m_tile * BLOCK_M, full);
                 if (dual && lane == 30) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * KB_ELEMS, BLOCK_M, full);  // second m-tile
@@ -468,41 +504,65 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int b0 = un.box_begin; b0 < un.box_end && ok; b0 += MAX_BOXES, ++tile) {
                 const int nb = min(MAX_BOXES, un.box_end - b0);
                 const uint32_t as = dual ? 0u : (tile & 1u), aphase = dual ? (tile & 1u) : ((tile >> 1) & 1u);
+                const int col0 = b0 * BOX_N;
+                const int n_valid = min(nb * BOX_N, p.V - col0);
+                // 8-bit mode: fetch the column scales of the whole tile while the tile is still being
+                // computed (lane l keeps the scale of column 32 c + l for each of the eight 32-column chunks)
+                float sc[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+                if (Q8) {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) sc[c] = (c * 32 + lane < n_valid) ? p.col_scale[col0 + c * 32 + lane] : 0.0f;
+                }
                 if (!mbar_wait(bar_tfull + 8 * as, aphase, abort_flag)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const int col0 = b0 * BOX_N;
-                const int n_valid = min(nb * BOX_N, p.V - col0);
-                for (int c = 0; c * 32 < n_valid; ++c) {
+                if (IS_ARGMAX) {
+                    // (the chunk loop stays rolled: it runs once per tile, and a short loop body that is
+                    // fetched once beats eight copies that are each fetched cold)
+                    auto sweep = [&](uint32_t acc_col, float& bv, int& bi) {
+                        for (int c = 0; c * 32 < n_valid; ++c) {
+                            uint32_t r[32];
+                            float v[32];
+                            float my_scale = sc[0];  // sc[c] by selection: keeps sc[] in registers
+                            if (Q8) {
+#pragma unroll
+                                for (int k = 1; k < 8; ++k) my_scale = (c == k) ? sc[k] : my_scale;
+                            }
+                            __syncwarp();
+                            tmem_ld32(lane_base + acc_col + c * 32, r);
+                            tmem_wait_ld();
+                            const int lim = n_valid - c * 32;  // >= 1
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                v[j] = __uint_as_float(r[j]);
+                                if (Q8) v[j] *= __shfl_sync(0xffffffffu, my_scale, j);
+                            }
+                            if (lim < 32) {  // ragged end of the vocabulary
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] = j < lim ? v[j] : -INFINITY;
+                            }
+                            float cv;
+                            int co;
+                            chunk_argmax(v, cv, co);
+                            if (cv > bv) {  // earlier chunks hold lower token ids: strict
+                                bv = cv;
+                                bi = col0 + c * 32 + co;
+                            }
+                        }
+                    };
+                    sweep(as * ACC_COLS, best_v, best_i);
+                    if (dual) sweep(ACC_COLS, best_v2, best_i2);
+                }
+                for (int c = 0; !IS_ARGMAX && c * 32 < n_valid; ++c) {
                     uint32_t r[32];
                     __syncwarp();
                     tmem_ld32(lane_base + as * ACC_COLS + c * 32, r);
                     tmem_wait_ld();
                     const int cbase = col0 + c * 32;
                     const int lim = n_valid - c * 32;  // >= 1
-                    if (MODE == MODE_ARGMAX) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const float v = __uint_as_float(r[j]);
-                            if (j < lim && v > best_v) {
-                                best_v = v;
-                                best_i = cbase + j;
-                            }
-                        }
-                    } else if (MODE == MODE_ARGMAX_Q8) {
-                        // lane j fetches the scale of column cbase + j once; the warp passes it round
-                        const float my_scale = lane < lim ? p.col_scale[cbase + lane] : 0.0f;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const float v = __uint_as_float(r[j]) * __shfl_sync(0xffffffffu, my_scale, j);
-                            if (j < lim && v > best_v) {
-                                best_v = v;
-                                best_i = cbase + j;
-                            }
-                        }
-                    } else if (MODE == MODE_TOPK) {
+                    if (MODE == MODE_TOPK) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             const float v = __uint_as_float(r[j]);
@@ -538,26 +598,6 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
                                 if (j < lim) out[j] = __uint_as_float(r[j]);
-                        }
-                    }
-                }
-                if (dual) {
-                    for (int c = 0; c * 32 < n_valid; ++c) {
-                        uint32_t r[32];
-                        __syncwarp();
-                        tmem_ld32(lane_base + ACC_COLS + c * 32, r);
-                        tmem_wait_ld();
-                        const int cbase = col0 + c * 32;
-                        const int lim = n_valid - c * 32;
-                        const float my_scale = Q8 && lane < lim ? p.col_scale[cbase + lane] : 1.0f;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            float v = __uint_as_float(r[j]);
-                            if (Q8) v *= __shfl_sync(0xffffffffu, my_scale, j);
-                            if (j < lim && v > best_v2) {
-                                best_v2 = v;
-                                best_i2 = cbase + j;
-                            }
                         }
                     }
                 }
@@ -774,17 +814,16 @@ static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks, bool all
     return s;
 }
 
-// Tensor map of the unembedding (or, for the unigram, the embedding) for the shape's box size,
-// encoded once per context.
-static int w_map(spec_ctx* ctx, const Shape& sh, const CUtensorMap** out, bool embedding = false) {
-    CUtensorMap* maps = embedding ? ctx->tm_e : ctx->tm_w;
-    bool* ready = embedding ? ctx->tm_e_ready : ctx->tm_w_ready;
-    if (!ready[sh.box_idx]) {
-        int rc = make_tensor_map(ctx, &maps[sh.box_idx], embedding ? ctx->embed : ctx->unembed, ctx->V, ctx->d, sh.box_n);
+// Tensor maps of the unembedding (or, for the unigram, the embedding), encoded once per context.
+static int w_map(spec_ctx* ctx, const WMaps** out, bool embedding = false) {
+    WMaps* maps = embedding ? &ctx->tm_e : &ctx->tm_w;
+    bool& ready = embedding ? ctx->tm_e_ready : ctx->tm_w_ready;
+    if (!ready) {
+        int rc = make_w_maps(ctx, maps, embedding ? ctx->embed : ctx->unembed, 2);
         if (rc) return rc;
-        ready[sh.box_idx] = true;
+        ready = true;
     }
-    *out = &maps[sh.box_idx];
+    *out = maps;
     return SPEC_OK;
 }
 
@@ -837,8 +876,8 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     int rc = set_smem_attr<MODE_ARGMAX, 1>(ctx);
     if (rc) return rc;
     const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
-    const CUtensorMap* tmW;
-    if ((rc = w_map(ctx, sh, &tmW))) return rc;
+    const WMaps* tmW;
+    if ((rc = w_map(ctx, &tmW))) return rc;
     const CUtensorMap* tmA;
     if ((rc = a_tensor_map(ctx, &tmA, d_hidden, M, ctx->d, sh.a_box_rows))) return rc;
     GemmParams p;
@@ -921,9 +960,9 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
     int rc = set_smem_attr<MODE_ARGMAX_Q8, 1>(ctx);
     if (rc) return rc;
     const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
-    if (!ctx->tm_q_ready[sh.box_idx]) {
-        if ((rc = make_tensor_map(ctx, &ctx->tm_q[sh.box_idx], ctx->wq, ctx->V, ctx->d, sh.box_n, 1))) return rc;
-        ctx->tm_q_ready[sh.box_idx] = true;
+    if (!ctx->tm_q_ready) {
+        if ((rc = make_w_maps(ctx, &ctx->tm_q, ctx->wq, 1))) return rc;
+        ctx->tm_q_ready = true;
     }
     const CUtensorMap* tmA;
     if ((rc = a_tensor_map(ctx, &tmA, d_hq, M, ctx->d, sh.a_box_rows, 1))) return rc;
@@ -935,7 +974,7 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
     p.col_scale = ctx->wscale;
     p.row_scale = d_hscale;
     cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX_Q8, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA,
-                               ctx->tm_q[sh.box_idx], p);
+                               ctx->tm_q, p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax_fp8 launch");
 }
@@ -944,8 +983,8 @@ int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cud
     int rc = set_smem_attr<MODE_STORE, 1>(ctx);
     if (rc) return rc;
     const Shape sh = cached_shape(ctx, m, (size_t)1 << 20);
-    const CUtensorMap* tmW;
-    if ((rc = w_map(ctx, sh, &tmW))) return rc;
+    const WMaps* tmW;
+    if ((rc = w_map(ctx, &tmW))) return rc;
     CUtensorMap tmA;
     if ((rc = make_tensor_map(ctx, &tmA, d_rows, m, ctx->d, sh.a_box_rows))) return rc;
     GemmParams p;
@@ -965,8 +1004,8 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
     // partial lists cost 8 bytes per entry and chunk: keep them under 256 MB
     int max_chunks = (int)std::max<long long>(1, (256ll << 20) / ((long long)V * k_tab * 8));
     const Shape sh = cached_shape(ctx, V, (size_t)max_chunks);
-    const CUtensorMap* tmW;
-    if ((rc = w_map(ctx, sh, &tmW))) return rc;
+    const WMaps* tmW;
+    if ((rc = w_map(ctx, &tmW))) return rc;
     CUtensorMap tmA;
     if ((rc = make_tensor_map(ctx, &tmA, d_rows, V, ctx->d, sh.a_box_rows))) return rc;
     const size_t need = (size_t)sh.n_chunks * V * k_tab;
@@ -1127,8 +1166,8 @@ int launch_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2,
     unigram_colsum_kernel<<<dim3((d + 127) / 128, n_slabs), 128, 0, st>>>(W, V, d, ctx->d_colsum);
     unigram_mean_kernel<<<(d + 127) / 128, 128, 0, st>>>(ctx->d_colsum, n_slabs, V, d, mean);
     unigram_centre_kernel<<<ctx->num_sms * 8, 256, 0, st>>>(W, mean, n, d, (__nv_bfloat16*)ctx->d_centred);
-    const CUtensorMap* tmE;
-    if ((rc = w_map(ctx, sh, &tmE, true))) return rc;
+    const WMaps* tmE;
+    if ((rc = w_map(ctx, &tmE, true))) return rc;
     CUtensorMap tmA;
     if ((rc = make_tensor_map(ctx, &tmA, ctx->d_centred, V, d, sh.a_box_rows))) return rc;
     GemmParams p;
