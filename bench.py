@@ -305,9 +305,18 @@ def main():
 
     fused = args.fuse      # measured equal on B200: dependent launch already hides the accept launch
 
-    def step(timers=None):
-        lens.copy_(lens0)                      # every iteration sees the same history length
+    # Every step sees the same history: step k of a round works on its own copy of the lengths, and one
+    # small copy per round of R steps restores all of them.  (A reset before every step would sit between
+    # accept and the next draft and break the dependent-launch chain that a real decode loop has there.)
+    R = max(r for r in range(1, 17) if args.steps % r == 0)
+    lens_all = lens0.unsqueeze(0).repeat(R, 1).contiguous()
+    lens0_all = lens_all.clone()
+    cfg["steps_per_replay"] = R
+
+    def step(timers=None, k=0):
+        lens = lens_all[k]
         if timers:
+            lens.copy_(lens0)
             timers[0].record()
         ctx.draft_context_ngrams(hist, lens, c["qs"], c["topk"], B, w, out=out_d)
         if timers:
@@ -328,28 +337,33 @@ def main():
         torch.cuda.synchronize()
 
     # The step is launch-bound at small sizes: capture it once in a CUDA graph and replay it.
+    def round_of_steps():
+        lens_all.copy_(lens0_all)
+        for k in range(R):
+            step(k=k)
+
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
         for _ in range(3):
-            step()
+            round_of_steps()
     torch.cuda.synchronize()
     graph = None
     if not args.no_graph:
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
-            step()
-    run_step = graph.replay if graph is not None else step
+            round_of_steps()
+    run_round = graph.replay if graph is not None else round_of_steps
     launches_per_step = 2 if (fused and S <= 256) else 3   # draft, verify(+accept) (the length reset is a torch copy)
 
-    for _ in range(args.warmup):
-        run_step()
+    for _ in range((args.warmup + R - 1) // R):
+        run_round()
     barrier()
     t_begin, t_end = ev(), ev()
     with ClockSampler(local_rank) as clk:
         barrier()
         t_begin.record()
-        for i in range(args.steps):
-            run_step()
+        for i in range(args.steps // R):
+            run_round()
         t_end.record()
         barrier()
     total_ms = t_begin.elapsed_time(t_end)

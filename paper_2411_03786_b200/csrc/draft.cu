@@ -164,6 +164,18 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     int32_t* hist_s = rep + P.hist_off;
 
     grid_launch_dependents();  // the verify kernel may start streaming weights while this one runs
+    // the first pass's empty table does not depend on the inputs: prepare it while the previous kernel drains
+    if (leader) {
+        for (int i = tid; i < P.slots; i += nthr) {
+            rep[i] = -1;
+            cnt[i] = 0;
+            last[i] = -1;
+        }
+        if (tid == 0) {
+            sm->n_groups = 0;
+            sm->overflow = 0;
+        }
+    }
     grid_dependency_wait();    // history and lengths come from the previous step's commit
     int L = P.len[s];
     if (L < 0 || L > P.cap) {
@@ -184,7 +196,11 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     if (tid < kMaxKTab) sm->chain_ok[tid] = 0;
     __syncthreads();
 
-    // ---- extended model bigram of the last token (rank r on lane r), overlapped with the scan
+    // ---- extended model bigram of the last token (rank r on lane r), overlapped with the scan: with a
+    // precomputed extension table the loads are only issued here and their values are picked up after
+    // the scan, so nobody waits for them at the barriers in between
+    int chain_tok[kMaxW];
+    bool chain_pending = false;
     if (leader && warp == nwarps - 1 && (P.flags & SPEC_FLAG_MODEL_FILL) && L >= 1) {
         const int x = sm->tq[0];
         if (x < 0 || x >= P.V) {
@@ -193,15 +209,9 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             bool ok = true;
             if (P.ext != nullptr && w <= P.w_ext) {
                 const int32_t* e = P.ext + ((size_t)x * P.k_tab + lane) * P.w_ext;
-                int t[kMaxW];  // all loads first, so they are in flight together
 #pragma unroll
-                for (int j = 0; j < kMaxW; ++j) t[j] = (j < w) ? e[j] : 0;
-#pragma unroll
-                for (int j = 0; j < kMaxW; ++j)
-                    if (j < w) {
-                        ok = ok && (t[j] >= 0 && t[j] < P.V);
-                        sm->chain[lane][j] = t[j];
-                    }
+                for (int j = 0; j < kMaxW; ++j) chain_tok[j] = (j < w) ? e[j] : 0;  // in flight together
+                chain_pending = true;
             } else {
                 int t = P.tab[(size_t)x * P.k_tab + lane];
                 for (int j = 0; j < w; ++j) {
@@ -213,8 +223,10 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                     t = P.tab[(size_t)t * P.k_tab];
                 }
             }
-            sm->chain_ok[lane] = ok ? 1 : 0;
-            if (!ok) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
+            if (!chain_pending) {
+                sm->chain_ok[lane] = ok ? 1 : 0;
+                if (!ok) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
+            }
         }
     }
 
@@ -233,7 +245,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         if (tid < kMaxNQ) sm->n_run[tid] = 0;
         bool overflowed = false;
         for (int r = 0; r < R && !overflowed; ++r) {
-            if (leader) {
+            if (leader && (R > 1 || r > 0)) {  // (the table of the very first pass was prepared at kernel entry)
                 for (int i = tid; i < P.slots; i += nthr) {
                     rep[i] = -1;
                     cnt[i] = 0;
@@ -397,6 +409,17 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         }
     }
     if (!leader) return;  // nobody reads a non-leader's shared memory, and no cluster barrier follows
+    if (chain_pending) {
+        bool ok = true;
+#pragma unroll
+        for (int j = 0; j < kMaxW; ++j)
+            if (j < w) {
+                ok = ok && (chain_tok[j] >= 0 && chain_tok[j] < P.V);
+                sm->chain[lane][j] = chain_tok[j];
+            }
+        sm->chain_ok[lane] = ok ? 1 : 0;
+        if (!ok) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
+    }
     __syncthreads();
 
     // ---- mixed allocation: context rows in query order, then model rows by rank; drop duplicates.
