@@ -26,42 +26,22 @@ __device__ __forceinline__ void accept_sequence(const AcceptArgs& q, int s, int 
     const int B = q.B, w = q.w;
     const int32_t* ds = q.drafts + (size_t)s * B * w;
     const int32_t* ps = q.argmax + (size_t)s * B * (w + 1);
-    // Everything the decision needs is requested up front, so the loads are in flight together: a
-    // compare-as-you-go loop would pay one memory round trip per accepted token.
     int nb = q.ndrafts[s];
-    const int L = q.len[s];
-    unsigned key = 0;  // (a << 8) | (255 - b): the maximum is the longest prefix, lowest row
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        const int b = lane + 32 * half;
-        if (b < B) {  // rows beyond ndrafts are read too (they hold -1) and ignored below
-            int dr[kMaxW], pr[kMaxW];
-#pragma unroll
-            for (int j = 0; j < kMaxW; ++j) {
-                dr[j] = j < w ? ds[b * w + j] : 0;
-                pr[j] = j < w ? ps[b * (w + 1) + j] : 1;
-            }
-            int a = 0;
-            bool run = true;
-#pragma unroll
-            for (int j = 0; j < kMaxW; ++j) {
-                run = run && j < w && dr[j] == pr[j];
-                a += run ? 1 : 0;
-            }
-            const int nbc = nb < 0 ? 0 : (nb > B ? B : nb);
-            if (b < nbc) {
-                unsigned k = ((unsigned)a << 8) | (unsigned)(255 - b);
-                key = k > key ? k : key;
-            }
-        }
-    }
     nb = nb < 0 ? 0 : (nb > B ? B : nb);
+    unsigned key = 0;  // (a << 8) | (255 - b): the maximum is the longest prefix, lowest row
+    for (int b = lane; b < nb; b += 32) {
+        int a = 0;
+        while (a < w && ds[b * w + a] == ps[b * (w + 1) + a]) ++a;
+        unsigned k = ((unsigned)a << 8) | (unsigned)(255 - b);
+        key = k > key ? k : key;
+    }
     key = __reduce_max_sync(0xffffffffu, key);
     int a = 0, b = 0;
     if (nb > 0) {
         a = (int)(key >> 8);
         b = 255 - (int)(key & 255u);
     }
+    const int L = q.len[s];
     const bool fits = (L >= 0) && (L + a + 1 <= q.cap);
     int32_t tok = -1;
     if (fits && lane <= a) tok = (lane < a) ? ds[b * w + lane] : ps[b * (w + 1) + a];

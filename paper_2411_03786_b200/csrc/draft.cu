@@ -196,11 +196,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     if (tid < kMaxKTab) sm->chain_ok[tid] = 0;
     __syncthreads();
 
-    // ---- extended model bigram of the last token (rank r on lane r), overlapped with the scan: with a
-    // precomputed extension table the loads are only issued here and their values are picked up after
-    // the scan, so nobody waits for them at the barriers in between
-    int chain_tok[kMaxW];
-    bool chain_pending = false;
+    // ---- extended model bigram of the last token (rank r on lane r), overlapped with the scan
     if (leader && warp == nwarps - 1 && (P.flags & SPEC_FLAG_MODEL_FILL) && L >= 1) {
         const int x = sm->tq[0];
         if (x < 0 || x >= P.V) {
@@ -209,9 +205,15 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             bool ok = true;
             if (P.ext != nullptr && w <= P.w_ext) {
                 const int32_t* e = P.ext + ((size_t)x * P.k_tab + lane) * P.w_ext;
+                int t[kMaxW];  // all loads first, so they are in flight together
 #pragma unroll
-                for (int j = 0; j < kMaxW; ++j) chain_tok[j] = (j < w) ? e[j] : 0;  // in flight together
-                chain_pending = true;
+                for (int j = 0; j < kMaxW; ++j) t[j] = (j < w) ? e[j] : 0;
+#pragma unroll
+                for (int j = 0; j < kMaxW; ++j)
+                    if (j < w) {
+                        ok = ok && (t[j] >= 0 && t[j] < P.V);
+                        sm->chain[lane][j] = t[j];
+                    }
             } else {
                 int t = P.tab[(size_t)x * P.k_tab + lane];
                 for (int j = 0; j < w; ++j) {
@@ -223,10 +225,8 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                     t = P.tab[(size_t)t * P.k_tab];
                 }
             }
-            if (!chain_pending) {
-                sm->chain_ok[lane] = ok ? 1 : 0;
-                if (!ok) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
-            }
+            sm->chain_ok[lane] = ok ? 1 : 0;
+            if (!ok) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
         }
     }
 
@@ -409,17 +409,6 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         }
     }
     if (!leader) return;  // nobody reads a non-leader's shared memory, and no cluster barrier follows
-    if (chain_pending) {
-        bool ok = true;
-#pragma unroll
-        for (int j = 0; j < kMaxW; ++j)
-            if (j < w) {
-                ok = ok && (chain_tok[j] >= 0 && chain_tok[j] < P.V);
-                sm->chain[lane][j] = chain_tok[j];
-            }
-        sm->chain_ok[lane] = ok ? 1 : 0;
-        if (!ok) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
-    }
     __syncthreads();
 
     // ---- mixed allocation: context rows in query order, then model rows by rank; drop duplicates.
