@@ -350,7 +350,8 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                     const unsigned long long mine = sm->gkey[g];
                     const int o_end = min(n_groups, (part + 1) * span);
                     int rank = 0;
-                    for (int o = part * span; o < o_end; ++o) {
+                    // a group with topk larger keys cannot be emitted: most groups (single occurrences) stop early
+                    for (int o = part * span; o < o_end && rank < P.topk; ++o) {
                         const unsigned long long other = sm->gkey[o];
                         rank += ((other >> 60) == (mine >> 60) && other > mine) ? 1 : 0;
                     }

@@ -118,3 +118,33 @@ def test_fp8_verify_full_size_C2(ngs):
             assert np.array_equal(am16.cpu().numpy(), am)
     assert ctx.get_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("name", ["C3", "C4"])
+def test_fp8_verify_full_size_sampled_rows(ngs, name):
+    """Tensor-bound launch shapes of the benchmark (several m-tiles, V=32000 and V=128256): all M rows on the GPU,
+    a seeded sample of rows (tile edges included) through the oracle."""
+    c = synth.config(name)
+    W = weights(c, "W")
+    ctx = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
+    wq, ws = ctx.quantize_head_fp8()
+    Wq, Ws = oracle.quantize_rows_e4m3(W)
+    assert np.array_equal(ws.cpu().numpy(), Ws)
+    g = synth.stream(c["seed"], "fp8/rows-checked")
+    M = c["M"]
+    rows = np.array(sorted({0, 1, 127, 128, M - 1, M - 2, (M - 1) // 128 * 128} | set(g.integers(0, M, 9).tolist())), dtype=np.int64)
+    assert np.array_equal(wq.cpu().numpy()[rows % c["V"]], Wq[rows % c["V"]])
+    H = synth.hidden_literal(M, c["d"], seed=c["seed"] + 8)
+    targets = g.integers(0, c["V"], M).astype(np.int32)
+    H[::2] = synth.hidden_planted(W, targets[::2], seed=c["seed"] + 9)      # every other row has a planted arg max
+    am, mx = ctx.verify_lmhead_argmax_fp8(dev_bf16(H), with_max=True)
+    am, mx = am.cpu().numpy(), mx.cpu().numpy().astype(np.float64)
+    Hq, Hs = oracle.quantize_rows_e4m3(H[rows])
+    ref_am, ref_mx, gap = oracle.verify_q8(Hq, Hs, Wq, Ws)
+    bad = am[rows] != ref_am
+    assert not (bad & (gap >= TOL)).any()
+    assert np.abs(mx[rows] - ref_mx).max() <= TOL
+    assert np.array_equal(am[::2], targets[::2])
+    assert am.min() >= 0 and am.max() < c["V"]
+    assert ctx.get_status() == 0
+    ctx.close()
