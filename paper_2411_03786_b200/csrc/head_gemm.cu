@@ -745,11 +745,13 @@ static void finish_shape(Shape& sh, int a_rows, int V) {
     sh.smem = sh.stages * sh.stage_bytes + pad + SMEM_MISC;
 }
 
-// Unit shapes.  One m-tile (memory-bound): every SM streams its own slice of W once, in 32-row
-// boxes so slices balance to within one box.  Several m-tiles (tensor-bound): `group` m-tiles
-// share each W chunk, W is loaded in 256-row boxes (one TMA issue per k-block) and every slot
-// sweeps one chunk per m-group.  (Measured on B200, V=32000, d=4096: 32-row boxes 0.9, 64-row
-// 1.1, 256-row 1.2 PFLOP/s; groups of 8..16 beat groups of 2..4 by 10-20%.)
+// Unit shapes.  `box_n` is the granularity in which the vocabulary is cut into chunks and tiles (a
+// tile is then copied in power-of-two pieces, see the producer).  One m-tile (memory-bound): every
+// SM streams its own slice of W once, cut to 32 rows so slices balance to within 32 rows.  Several
+// m-tiles (tensor-bound): `group` m-tiles share each W chunk, tiles are whole 256-row blocks (one
+// copy per k-block) and every slot sweeps one chunk per m-group.  (Measured on B200, V=32000,
+// d=4096, when a tile was still copied box by box: 32-row boxes 0.9, 64-row 1.1, 256-row
+// 1.2 PFLOP/s; groups of 8..16 beat groups of 2..4 by 10-20%.)
 static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks, bool allow_dual) {
     const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
     Shape sh{};
