@@ -14,6 +14,8 @@
  *     After an error spec_last_error() gives a one-line reason.
  *   - Pointers named d_* are DEVICE pointers owned by the caller, 16-byte aligned, and must stay
  *     valid until the stream work that uses them has finished.  Other pointers are host pointers.
+ *     (Any device-accessible address works: small outputs such as d_acc_len / d_committed may live in
+ *     mapped pinned host memory, which saves the caller a device-to-host copy per step.)
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All calls are
  *     asynchronous with respect to the host except spec_init, spec_destroy and spec_get_status.
  *   - Tokens are int32 in [0, V).  A history matrix is hist[S, cap] (row stride cap, cap % 4 == 0)

@@ -76,7 +76,9 @@ def load_library(build: bool = True) -> C.CDLL:
 def _ptr(t, dtype=None):
     if t is None:
         return None
-    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    # pinned host memory is mapped into the device address space (unified addressing): small outputs may
+    # live there so that a kernel's result reaches the host without a separate copy
+    assert (t.is_cuda or t.is_pinned()) and t.is_contiguous(), "tensors must be contiguous CUDA (or pinned host) tensors"
     if dtype is not None:
         assert t.dtype == dtype, f"expected {dtype}, got {t.dtype}"
     return C.c_void_p(t.data_ptr())
