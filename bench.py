@@ -508,6 +508,67 @@ def main():
     d2h = out_a2[0].numel() * 4 + out_a2[2].numel() * 4        # what the kernel stores into host memory per step
     assert torch.equal(out_a2[0], out_a[0].cpu()), "the host copy of the accepted lengths differs from the device run"
 
+    # ---- the same end-to-end step, two deep: step i+1's uploads run while step i computes, and the host reads
+    # step i's result while step i+1 is already queued (how a serving loop would drive it).  Extra information:
+    # the e2e value above stays the one-step-at-a-time figure.
+    pipe_ms = None
+    if graph is not None and rank == 0 and world == 1:
+        sets = []
+        for bset in range(2):
+            ht, hh, ho = pinned(tok_specs), pinned(hid_specs), pinned(out_specs)
+            dt, dh = ondev(tok_specs), ondev(hid_specs)
+            ht.copy_(h_tok); hh.copy_(h_hid)
+            dhist, dlens = carve(dt, tok_specs)
+            (dHb,) = carve(dh, hid_specs)
+            outb = (carve(ho, out_specs)[0], out_a[1], carve(ho, out_specs)[1])
+
+            def compute(dhist=dhist, dlens=dlens, dHb=dHb, outb=outb):
+                ctx.draft_context_ngrams(dhist, dlens, c["qs"], c["topk"], B, w, out=out_d)
+                if fused:
+                    ctx.verify_accept_commit(dHb, out_d[0], out_d[1], dhist, dlens, argmax=out_v[0], out=outb)
+                else:
+                    ctx.verify_lmhead_argmax(dHb, out=out_v)
+                    ctx.accept_and_commit(out_d[0], out_d[1], out_v[0].view(S, B, w + 1), dhist, dlens, out=outb)
+
+            with torch.cuda.stream(side):
+                dt.copy_(ht); dh.copy_(hh)
+                compute()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                compute()
+            sets.append(dict(ht=ht, hh=hh, ho=ho, dt=dt, dh=dh, g=g, acc=outb[0], up=torch.cuda.Event(), done=torch.cuda.Event()))
+        main = torch.cuda.current_stream()
+
+        def pipelined(n):
+            tokens = 0
+            for i in range(n):
+                cur, prev = sets[i & 1], sets[(i & 1) ^ 1]
+                if i >= 2:
+                    copy_stream.wait_event(cur["done"])       # the step that used these device buffers has finished
+                with torch.cuda.stream(copy_stream):
+                    cur["dt"].copy_(cur["ht"], non_blocking=True)
+                    cur["dh"].copy_(cur["hh"], non_blocking=True)
+                    cur["up"].record(copy_stream)
+                main.wait_event(cur["up"])
+                cur["g"].replay()
+                cur["done"].record(main)
+                if i >= 1:
+                    prev["done"].synchronize()
+                    tokens += int(prev["acc"].sum()) + S       # the host reads the previous step's result
+            sets[(n - 1) & 1]["done"].synchronize()
+            return tokens + int(sets[(n - 1) & 1]["acc"].sum()) + S
+
+        pipelined(20)
+        torch.cuda.synchronize()
+        p0, p1 = ev(), ev()
+        p0.record()
+        tok_pipe = pipelined(args.steps)
+        p1.record()
+        torch.cuda.synchronize()
+        pipe_ms = p0.elapsed_time(p1) / args.steps
+        assert tok_pipe == int(round(acc_mean)) * args.steps, "the pipelined loop committed a different number of tokens"
+
     # ---- max over ranks, totals over ranks
     from paper_2411_03786_b200.multigpu import reduce_max_sum
     (total_ms, e2e_ms, verify_ms, verify_alone_ms), (acc_total,) = reduce_max_sum(
@@ -556,7 +617,8 @@ def main():
                 "steps_per_s": world * 1e3 / ms_per_step, "tokens_per_step": acc_total / world / S,
                 "phase_ms": {"draft": draft_ms, "verify": verify_ms, "accept": accept_ms},
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                        "ms_per_step": e2e_ms / args.steps},
+                        "ms_per_step": e2e_ms / args.steps, "mode": "one step at a time: upload, step, host waits for the result",
+                        "pipelined_two_deep_ms_per_step": pipe_ms},
                 "gpu_launches": int(launches) * world, "launch_mode": "eager" if graph is None else "cuda_graph_replay", "roofline": roof, "table_build": table, "cpu_baseline": cpu,
                 "clocks": clk.summary(), "status_bits": status, "copied_fraction": copied}
         if fp8:
