@@ -221,6 +221,14 @@ def test_fused_verify_accept_equals_the_two_calls_and_the_oracle(ngs, S, B, w):
     assert np.array_equal(acc2.cpu().numpy(), acc_r) and np.array_equal(best2.cpu().numpy(), best_r)
     assert np.array_equal(com2.cpu().numpy(), com_r) and np.array_equal(h2.cpu().numpy(), h_ref)
     assert np.array_equal(l2.cpu().numpy(), l_ref)
+    # small outputs may live in mapped pinned host memory: the kernel's stores are the device-to-host transfer
+    pin = lambda *shape: torch.full(shape, -9, dtype=torch.int32).pin_memory()
+    out3 = (pin(S), pin(S), pin(S, w + 1))
+    h3, l3 = dev_i32(hist), dev_i32(lens)
+    ctx.verify_accept_commit(dH, dD, dN, h3, l3, out=out3)
+    torch.cuda.synchronize()
+    assert np.array_equal(out3[0].numpy(), acc_r) and np.array_equal(out3[1].numpy(), best_r)
+    assert np.array_equal(out3[2].numpy(), com_r) and np.array_equal(h3.cpu().numpy(), h_ref)
     ctx.get_status()
     ctx.close()
 
