@@ -615,7 +615,8 @@ def main():
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16", "data": "synthetic", "config": cfg,
                 "steps_per_s": world * 1e3 / ms_per_step, "tokens_per_step": acc_total / world / S,
-                "phase_ms": {"draft": draft_ms, "verify": verify_ms, "accept": accept_ms},
+                "phase_ms": {"draft": draft_ms, "verify": verify_ms, "accept": accept_ms,
+                             "note": "events between eagerly launched calls: small kernels include the host's launch gap"},
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms / args.steps, "mode": "one step at a time: upload, step, host waits for the result",
                         "pipelined_two_deep_ms_per_step": pipe_ms},
