@@ -222,10 +222,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU work for the oracle baseline")
     ap.add_argument("--no-table", action="store_true", help="skip timing the one-off table build")
-    ap.add_argument("--scaled", action="store_true", help="also time draft/accept on bandwidth-sized batches")
+    ap.add_argument("--no-scaled", action="store_true", help="skip timing draft/accept on bandwidth-sized batches")
     ap.add_argument("--no-fuse", action="store_true",
                     help="call verify_lmhead_argmax and accept_and_commit separately instead of verify_accept_commit (one launch)")
-    ap.add_argument("--fp8", action="store_true", help="also time the 8-bit (E4M3) verification head; reported beside the bf16 numbers")
+    ap.add_argument("--fp8", action="store_true", help=argparse.SUPPRESS)      # accepted for older command lines: now the default
+    ap.add_argument("--scaled", action="store_true", help=argparse.SUPPRESS)   # likewise
+    ap.add_argument("--no-fp8", action="store_true", help="skip timing the 8-bit (E4M3) verification head (reported beside the bf16 numbers)")
     ap.add_argument("--no-graph", action="store_true", help="launch the step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -411,7 +413,7 @@ def main():
     verify_alone_ms = verify_eager_ms if verify_graph_ms is None else min(verify_eager_ms, verify_graph_ms)
 
     fp8 = None
-    if args.fp8 and c["d"] % 16 == 0:
+    if not args.no_fp8 and c["d"] % 16 == 0:
         # quantise the head once, then the same back-to-back timing: each call = quantise H (1 launch) + contraction
         ctx.quantize_head_fp8()
         scratch8 = (torch.empty((M, c["d"]), dtype=torch.uint8, device=dev), torch.empty(M, dtype=torch.float32, device=dev))
@@ -593,7 +595,7 @@ def main():
                  "timing": "CUDA events around back-to-back launches on the launching stream (the faster of eager launches and one graph replay)", "algorithmic_bytes": bytes_alg, "flops": flops,
                  "peak_source": pk["source"] + (" sustained" if roof["bound"] == "tensor" else " copy")})
 
-    scaled = scaled_streams(ctx, torch, dev, c, pk) if (args.scaled and rank == 0) else None
+    scaled = scaled_streams(ctx, torch, dev, c, pk) if (not args.no_scaled and rank == 0 and world == 1) else None
     line = None
     if rank == 0:
         cpu = {}
