@@ -74,10 +74,12 @@ def test_fp8_exact_ties_take_the_lowest_token(ngs):
     V, d = 700, 128
     W = synth.gaussian_weights(V, d, 1.0, 9, "W")
     W[[40, 300, 650]] = W[5]
+    W[[6, 9, 17, 31]] = W[5]               # ties inside one 32-column chunk, at every level of its comparison tree
+    W[[101, 99, 110]] = W[98]
     ctx = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
     ctx.quantize_head_fp8()
-    am, _ = ctx.verify_lmhead_argmax_fp8(dev_bf16(W[[5, 650]].copy()))
-    assert am.cpu().tolist() == [5, 5]
+    am, _ = ctx.verify_lmhead_argmax_fp8(dev_bf16(W[[5, 650, 110, 31]].copy()))
+    assert am.cpu().tolist() == [5, 5, 98, 5]
     ctx.close()
 
 

@@ -58,10 +58,12 @@ def test_verify_exact_ties_take_the_lowest_token(ngs):
     V, d = 700, 64
     W = synth.gaussian_weights(V, d, 1.0, 9, "W")
     W[[40, 300, 650]] = W[5]               # identical rows in different tiles / chunks
+    W[[6, 9, 17, 31]] = W[5]               # and inside one 32-column chunk, at every level of its comparison tree
+    W[[101, 99, 110]] = W[98]
     ctx = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
-    H = W[[5, 650]].copy()
+    H = W[[5, 650, 110, 31]].copy()
     am, _ = ctx.verify_lmhead_argmax(dev_bf16(H))
-    assert am.cpu().tolist() == [5, 5]
+    assert am.cpu().tolist() == [5, 5, 98, 5]
     ctx.close()
 
 
