@@ -66,10 +66,13 @@ struct GemmParams {
     int n_groups;  // ceil(n_mtiles / group)
     int n_slots;   // grid = group * n_slots
     int a_box_rows;   // rows of A per TMA box (128, or fewer when A has fewer rows)
+    int a2_rows;      // dual: rows of the second m-tile's TMA box (its own tensor map)
     int a_bytes;      // shared-memory bytes reserved for the A tile of a stage (multiple of 1024)
     int stage_bytes;  // a_bytes + boxes per tile * box bytes
+    int pad_bytes;    // unused bytes after the last stage (keeps the MMA's 128-row A window in bounds)
     int stages;       // depth of the operand ring
     int dual;         // 1: A has two m-tiles and every CTA computes both against its W slice (argmax only)
+    int tile2_m64;    // dual, and the second m-tile has at most 64 rows: it is computed with M = 64 instructions
     unsigned long long* keys;
     unsigned int* ticket;
     int32_t* argmax;
@@ -301,7 +304,8 @@ struct KbCursor {
 // KT = capacity of the per-thread top-k list (registers); only MODE_TOPK uses it.
 template <int MODE, int KT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ WMaps tmB, const GemmParams p) {
+head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA2,
+                 const __grid_constant__ WMaps tmB, const GemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;               // operand stages, 1024-byte aligned
@@ -310,7 +314,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int BOX_N = p.box_n, MAX_BOXES = TILE_N / p.box_n;
     // The MMA always reads a 128-row A tile; when fewer rows are loaded the rest of that window is
     // whatever follows in shared memory (rows that no output uses), so keep the window in bounds.
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES + (A_TILE_BYTES - A_BYTES));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + STAGES * STAGE_BYTES + p.pad_bytes);
     // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * MAX_STAGES;
@@ -327,6 +331,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (warp == 0 && lane < 6)  // the descriptors' first use would otherwise pay their fetch on the critical path
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(lane < 5 ? &tmB.m[lane] : &tmA)) : "memory");
+    if (IS_ARGMAX && p.dual && warp == 0 && lane == 6) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA2)) : "memory");
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -361,7 +366,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             long long issued = 0;
             bool ok = true;
             const bool dual = IS_ARGMAX && p.dual;
-            const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * BLOCK_K * 2 * (dual ? 2u : 1u);
+            const uint32_t a_box_bytes = (uint32_t)(p.a_box_rows + (dual ? p.a2_rows : 0)) * 128u;
             const int my_rows = 256 >> lane;  // lanes 0..4: the piece size this lane copies
             // piece of `rows` (a multiple of 16, at most 256) for this lane: the rows above it come first
             auto w_piece = [&](uint32_t sa, int kb, int b0, int nb, uint32_t full) {
@@ -396,7 +401,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     w_piece(sa, cur.kb, cur.b0, cur.nb, full);
                 }
                 if (lane == 31) tma_load_2d(sa, &tmA, cur.kb * KB_ELEMS, cur.un.m_tile * BLOCK_M, full);
-                if (dual && lane == 30) tma_load_2d(sa + A_TILE_BYTES, &tmA, cur.kb * KB_ELEMS, BLOCK_M, full);  // second m-tile
+                if (dual && lane == 30) tma_load_2d(sa + A_TILE_BYTES, &tmA2, cur.kb * KB_ELEMS, BLOCK_M, full);  // second m-tile
                 ++issued;
                 if (++stage == STAGES) {
                     stage = 0;
@@ -456,10 +461,12 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                         if (dual) {  // the same W tile against the second m-tile, into the other accumulator
                             const uint64_t adesc2 = make_kmajor_sw128_desc(sa + A_TILE_BYTES);
+                            // a second tile of at most 64 rows takes the M = 64 form: half the tensor work
+                            const uint32_t idesc2 = p.tile2_m64 ? ((idesc & ~(0x1Fu << 24)) | ((uint32_t)(64 >> 4) << 24)) : idesc;
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
-                                if (Q8) tc_mma_e4m3(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                                else tc_mma_bf16(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                                if (Q8) tc_mma_e4m3(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc2, (kb | k) != 0 ? 1u : 0u);
+                                else tc_mma_bf16(d_tmem + ACC_COLS, adesc2 + 2 * k, bdesc + 2 * k, idesc2, (kb | k) != 0 ? 1u : 0u);
                             }
                         }
                         tc_commit(bar_empty + 8 * stage);  // frees the stage once these MMAs have read it
@@ -606,10 +613,15 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * as);
             }
             if (!ok) break;
-            if (dual && row + BLOCK_M < p.a_rows) {
-                const unsigned long long key =
-                    ((unsigned long long)orderable_f32(best_v2) << 32) | (unsigned long long)(~(uint32_t)best_i2);
-                atomicMax(p.keys + row + BLOCK_M, key);
+            if (dual) {
+                // An M = 64 accumulator keeps row i in TMEM lane 32 (i / 16) + i % 16 (measured): the lower 16
+                // lanes of each epilogue warp hold rows, the upper 16 nothing.
+                const int row2 = BLOCK_M + (p.tile2_m64 ? quad * 16 + lane : row_in_tile);
+                if (row2 < p.a_rows && (!p.tile2_m64 || lane < 16)) {
+                    const unsigned long long key =
+                        ((unsigned long long)orderable_f32(best_v2) << 32) | (unsigned long long)(~(uint32_t)best_i2);
+                    atomicMax(p.keys + row2, key);
+                }
             }
             if (row < p.a_rows) {
                 if (IS_ARGMAX) {
@@ -725,7 +737,7 @@ __global__ void extend_table_kernel(const int32_t* __restrict__ tab, int V, int 
 // ------------------------------------------------------------------------------------------ host: unit shapes
 struct Shape {
     int box_n, box_idx, group, n_groups, n_slots, n_chunks, grid;
-    int a_box_rows, a_bytes, stage_bytes, stages, smem, dual;
+    int a_box_rows, a2_rows, a_bytes, stage_bytes, pad_bytes, stages, smem, dual;
 };
 
 // Derives the shared-memory geometry from (box_n, group, n_chunks, grid).
@@ -738,10 +750,14 @@ static void finish_shape(Shape& sh, int a_rows, int V) {
     const int chunk_max = (n_boxes + sh.n_chunks - 1) / sh.n_chunks;
     const int nb_max = std::min(TILE_N / sh.box_n, chunk_max);
     sh.a_box_rows = n_mtiles == 1 ? std::min(BLOCK_M, (a_rows + 7) / 8 * 8) : BLOCK_M;
-    sh.a_bytes = sh.dual ? 2 * A_TILE_BYTES : (sh.a_box_rows * BLOCK_K * 2 + 1023) / 1024 * 1024;
+    // dual: the second m-tile is loaded only as tall as it is (a smaller stage means a deeper ring)
+    sh.a2_rows = sh.dual ? std::min(BLOCK_M, (a_rows - BLOCK_M + 7) / 8 * 8) : 0;
+    const int a_last_bytes = ((sh.dual ? sh.a2_rows : sh.a_box_rows) * 128 + 1023) / 1024 * 1024;
+    sh.a_bytes = sh.dual ? A_TILE_BYTES + a_last_bytes : a_last_bytes;
     sh.stage_bytes = sh.a_bytes + (nb_max * sh.box_n * BLOCK_K * 2 + 1023) / 1024 * 1024;
-    const int pad = sh.dual ? 0 : A_TILE_BYTES - sh.a_bytes;
+    const int pad = A_TILE_BYTES - a_last_bytes;  // the MMA's 128-row window over the last A tile stays in bounds
     sh.stages = std::min(MAX_STAGES, (SMEM_LIMIT - SMEM_MISC - pad) / sh.stage_bytes);
+    sh.pad_bytes = pad;
     sh.smem = sh.stages * sh.stage_bytes + pad + SMEM_MISC;
 }
 
@@ -846,6 +862,7 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.num_kb = (ctx->d + BLOCK_K - 1) / BLOCK_K;
     p.n_mtiles = sh.dual ? 1 : (a_rows + BLOCK_M - 1) / BLOCK_M;  // dual: one unit covers both m-tiles
     p.dual = sh.dual;
+    p.tile2_m64 = (sh.dual && a_rows - BLOCK_M <= 64) ? 1 : 0;
     p.box_n = sh.box_n;
     p.n_boxes = (ctx->V + sh.box_n - 1) / sh.box_n;
     p.n_chunks = sh.n_chunks;
@@ -853,8 +870,10 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.n_groups = sh.n_groups;
     p.n_slots = sh.n_slots;
     p.a_box_rows = sh.a_box_rows;
+    p.a2_rows = sh.a2_rows;
     p.a_bytes = sh.a_bytes;
     p.stage_bytes = sh.stage_bytes;
+    p.pad_bytes = sh.pad_bytes;
     p.stages = sh.stages;
     p.keys = ctx->d_keys;
     p.ticket = ctx->d_ticket;
@@ -882,6 +901,8 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     if ((rc = w_map(ctx, &tmW))) return rc;
     const CUtensorMap* tmA;
     if ((rc = a_tensor_map(ctx, &tmA, d_hidden, M, ctx->d, sh.a_box_rows))) return rc;
+    const CUtensorMap* tmA2 = tmA;  // second m-tile of the two-tile pass: same matrix, a box only as tall as that tile
+    if (sh.dual && (rc = a_tensor_map(ctx, &tmA2, d_hidden, M, ctx->d, sh.a2_rows))) return rc;
     GemmParams p;
     fill_common(ctx, p, M, sh);
     p.argmax = d_argmax;
@@ -893,7 +914,7 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
     }
     p.keys_out = d_keys_out;
     p.idx_offset = idx_offset;
-    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA, *tmW, p);
+    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA, *tmA2, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax launch");
 }
@@ -968,6 +989,8 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
     }
     const CUtensorMap* tmA;
     if ((rc = a_tensor_map(ctx, &tmA, d_hq, M, ctx->d, sh.a_box_rows, 1))) return rc;
+    const CUtensorMap* tmA2 = tmA;
+    if (sh.dual && (rc = a_tensor_map(ctx, &tmA2, d_hq, M, ctx->d, sh.a2_rows, 1))) return rc;
     GemmParams p;
     fill_common(ctx, p, M, sh);
     p.num_kb = (ctx->d + BLOCK_K_Q8 - 1) / BLOCK_K_Q8;
@@ -975,7 +998,7 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
     p.maxv = d_max;
     p.col_scale = ctx->wscale;
     p.row_scale = d_hscale;
-    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX_Q8, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA,
+    cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX_Q8, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA, *tmA2,
                                ctx->tm_q, p);
     ctx->launches += 1;
     return check_cuda(ctx, e, "verify_lmhead_argmax_fp8 launch");
@@ -992,7 +1015,7 @@ int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cud
     GemmParams p;
     fill_common(ctx, p, m, sh);
     p.logits = d_logits;
-    head_gemm_kernel<MODE_STORE, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
+    head_gemm_kernel<MODE_STORE, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, tmA, *tmW, p);
     ctx->launches += 1;
     return check_cuda(ctx, cudaGetLastError(), "spec_debug_logits launch");
 }
@@ -1028,11 +1051,11 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
     p.part_val = ctx->d_part_val;
     p.part_idx = ctx->d_part_idx;
     if (kt == 8)
-        head_gemm_kernel<MODE_TOPK, 8><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
+        head_gemm_kernel<MODE_TOPK, 8><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, tmA, *tmW, p);
     else if (kt == 16)
-        head_gemm_kernel<MODE_TOPK, 16><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
+        head_gemm_kernel<MODE_TOPK, 16><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, tmA, *tmW, p);
     else
-        head_gemm_kernel<MODE_TOPK, 32><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmW, p);
+        head_gemm_kernel<MODE_TOPK, 32><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, tmA, *tmW, p);
     if ((rc = check_cuda(ctx, cudaGetLastError(), "build_model_ngram_tables launch"))) return rc;
     merge_topk_kernel<<<(V + 127) / 128, 128, 0, st>>>(ctx->d_part_val, ctx->d_part_idx, sh.n_chunks, V, k_tab, d_tab_idx,
                                                       d_tab_val);
@@ -1175,7 +1198,7 @@ int launch_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2,
     GemmParams p;
     fill_common(ctx, p, V, sh);
     p.part_val = ctx->d_part_val;
-    head_gemm_kernel<MODE_SUMSQ, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, *tmE, p);
+    head_gemm_kernel<MODE_SUMSQ, 1><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, tmA, *tmE, p);
     unigram_sum_kernel<<<(V + 255) / 256, 256, 0, st>>>(ctx->d_part_val, sh.n_chunks, V, d_dist2);
     ctx->launches += 5;
     if (k_uni > 0) {
