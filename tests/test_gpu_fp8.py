@@ -44,7 +44,8 @@ def test_quantiser_is_bit_exact(ngs, n, d):
 
 # one tile, ragged V / K tails (d % 128 != 0), two m-tiles in one pass, several m-tiles
 SHAPES = [(1024, 128, 20), (1000, 208, 150), (4136, 320, 300), (96, 64, 1), (33, 16, 129), (4136, 320, 256), (9000, 144, 200),
-          (5000, 4096, 200), (2100, 2048, 130)]                      # two m-tiles in one pass, k-loop longer than the ring
+          (5000, 4096, 200), (2100, 2048, 130),                      # two m-tiles in one pass, k-loop longer than the ring
+          (40000, 256, 200), (40000, 2048, 140), (40000, 512, 60)]    # ... and more than one 256-column tile per CTA
 
 
 @pytest.mark.parametrize("V,d,M", SHAPES)

@@ -25,7 +25,8 @@ def make_ctx(ngs, V, d, seed, std=1.0):
 
 # sizes span one tile, several tiles, ragged M / V / K tails
 SHAPES = [(1024, 128, 20), (1000, 200, 150), (4136, 320, 300), (96, 64, 1), (33, 8, 129), (4136, 320, 256), (9000, 128, 200),
-          (5000, 2048, 200), (2100, 1536, 130), (3000, 1024, 256)]   # two m-tiles in one pass, k-loop longer than the ring
+          (5000, 2048, 200), (2100, 1536, 130), (3000, 1024, 256),   # two m-tiles in one pass, k-loop longer than the ring
+          (40000, 256, 200), (40000, 1024, 140), (40000, 512, 60)]    # ... and more than one 256-column tile per CTA
 
 
 @pytest.mark.parametrize("V,d,M", SHAPES)
