@@ -25,7 +25,7 @@ def test_noalloc_verify_matches_context_verify_on_two_calls_in_a_row():
     W = synth.gaussian_weights(V, d, d ** -0.5, 21, "W")
     dW = dev_bf16(W)
     ctx = ngs.SpecContext(dW, dW)
-    for call, M in enumerate((300, 77)):   # second call reuses the scratch the first one left behind
+    for call, M in enumerate((300, 77, 200)):   # later calls reuse the scratch the earlier ones left behind; all three row regimes
         dH = dev_bf16(synth.hidden_literal(M, d, seed=50 + call))
         ref_am, ref_mx = ctx.verify_lmhead_argmax(dH, with_max=True)
         out = (torch.empty(M, dtype=torch.int32, device="cuda"), torch.empty(M, dtype=torch.float32, device="cuda"))
