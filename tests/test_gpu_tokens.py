@@ -187,7 +187,7 @@ def test_toy_model_decode_is_lossless_and_fully_accepted(ngs):
     ctx.close()
 
 
-@pytest.mark.parametrize("S,B,w", [(1, 8, 5), (7, 4, 3), (64, 16, 8), (300, 2, 2)])
+@pytest.mark.parametrize("S,B,w", [(1, 8, 5), (7, 4, 3), (64, 16, 8), (300, 2, 2), (5, 8, 4)])
 def test_fused_verify_accept_equals_the_two_calls_and_the_oracle(ngs, S, B, w):
     V, d = 777, 96
     g = np.random.default_rng(S * 100 + B)
