@@ -80,7 +80,7 @@ def test_draft_random_small_alphabets_and_ragged_lengths(ngs, small_ctx):
     assert small_ctx.get_status() == 0
 
 
-@pytest.mark.parametrize("L", [20000, 70000])      # one CTA per sequence / a cluster of four
+@pytest.mark.parametrize("L", [6000, 20000, 70000])      # history staged in shared memory / one CTA per sequence / a cluster of four
 def test_draft_many_distinct_continuations_uses_the_exact_multi_pass_path(ngs, small_ctx, L):
     # q = 1 on a two-token-heavy history: thousands of distinct continuations, more than the
     # shared-memory table holds in one pass.
