@@ -1,0 +1,56 @@
+"""GPU parity of the drafting kernel over seeded random problems: history lengths on both sides of every
+launch-shape threshold (thread count, staging in shared memory, clusters), alphabets from 2 symbols to the
+whole vocabulary, copy spans, every flag combination, with and without the precomputed extension table."""
+import numpy as np
+import pytest
+
+import oracle
+import synth
+from gpu_util import dev_bf16, dev_i32
+
+pytestmark = pytest.mark.gpu
+V = 512
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2411_03786_b200 as ngs
+    W = synth.gaussian_weights(V, 64, 1.0, 1, "W")
+    c = ngs.SpecContext(dev_bf16(W), dev_bf16(W))
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("case", range(48))
+def test_random_draft_problem(ctx, case):
+    import paper_2411_03786_b200 as ngs
+    g = np.random.default_rng(9000 + case)
+    S = int(g.integers(1, 7))
+    Lmax = int([g.integers(1, 64), g.integers(64, 2100), g.integers(2000, 8300), g.integers(8000, 17000),
+                g.integers(16000, 70000), g.integers(8100, 8300)][case % 6])
+    cap = (Lmax + int(g.integers(0, 200)) + 3) // 4 * 4
+    alpha = int(g.choice([2, 3, 6, 40, V]))
+    lens = np.array([Lmax if s == 0 else int(g.integers(0, Lmax + 1)) for s in range(S)], np.int32)
+    hist = np.full((S, cap), -1, np.int32)
+    for s in range(S):
+        h = g.integers(0, alpha, lens[s])
+        if g.random() < 0.5 and lens[s] > 40:
+            for _ in range(int(lens[s]) // 50):
+                a, b, n = int(g.integers(0, lens[s] - 20)), int(g.integers(0, lens[s] - 20)), int(g.integers(4, 20))
+                h[b:b + n] = h[a:a + n]
+        hist[s, :lens[s]] = h
+    n_q = int(g.integers(0, 4))
+    qs = [int(q) for q in g.choice([1, 2, 3, 4], n_q, replace=False)]
+    B = int(g.integers(1, 33))
+    w = int(g.integers(1, 12))
+    topk = int(g.integers(1, B + 1))
+    k_tab = int(g.integers(1, 17))
+    flags = int(g.choice([0, 1, 2, 3, 7, 5])) | (ngs.flag_reserve(int(g.integers(0, B + 1))) if g.random() < 0.3 else 0)
+    T = np.stack([g.permutation(V)[:k_tab] for _ in range(V)]).astype(np.int32)
+    ext = oracle.extend_table(T, w) if g.random() < 0.5 else None
+    ctx.set_model_table(dev_i32(T), dev_i32(ext) if ext is not None else None)
+    want = oracle.draft_batch(hist, lens, qs, topk, B, w, flags, T)
+    got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, flags)
+    for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
+        assert np.array_equal(a.cpu().numpy(), b), name
+    assert ctx.get_status() == 0
