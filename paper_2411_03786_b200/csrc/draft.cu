@@ -14,6 +14,11 @@
 // A history of up to 8192 tokens is first copied into shared memory (one round of 128-bit loads);
 // the scan, the key comparisons and the candidate rows then never wait for global memory again,
 // which is what the latency of a single short sequence is made of.
+//
+// The scan itself only looks for matches: per 128-bit vector one comparison chain, per warp iteration
+// (512 tokens) one vote.  Where a match turns up its position goes into a per-warp queue, and a
+// queue-full of matches is grouped at once, one per lane, so that the dependent reads each match
+// needs (suffix, continuation, the group's representative) overlap instead of stalling the scan.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -43,11 +48,13 @@ struct DraftParams {
     int max_groups;  // slots / 2
     int stage_hist;  // 1: copy the history into shared memory first (single CTA, short history)
     int hist_off;    // where that copy lives, in ints from the start of the hash table
+    int queue_off;   // byte offset of the per-warp match queues from the start of dynamic shared memory
 };
 
 constexpr int kMaxPasses = 1024;
 constexpr int kRankMax = 512;                          // groups ranked by counting (all threads) up to here
 constexpr int kMaxCand = kMaxNQ * kMaxB + kMaxKTab;    // candidate rows before duplicates are dropped
+constexpr int kMatchQueue = 128;                       // matches a warp queues before it groups them
 
 __device__ __forceinline__ uint32_t fmix32(uint32_t h) {
     h ^= h >> 16;
@@ -130,6 +137,10 @@ __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int 
     sm->overflow = 1;
 }
 
+// STREAM = false: the history was staged in shared memory (one CTA, short history; the latency of this
+// instantiation is a step's drafting latency, so it carries nothing it does not execute).
+// STREAM = true: the history is read from global memory, by one CTA or by a cluster.
+template <bool STREAM>
 __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DraftSmem* sm = reinterpret_cast<DraftSmem*>(smem_raw);
@@ -144,11 +155,13 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     cg::cluster_group cluster = cg::this_cluster();
     const int csize = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
     const bool leader = crank == 0;
-    DraftSmem* lsm = cluster.map_shared_rank(sm, 0);
-    int* lrep = cluster.map_shared_rank(rep, 0);
-    int* lcnt = cluster.map_shared_rank(cnt, 0);
-    int* llast = cluster.map_shared_rank(last, 0);
-    int* lgrp_slot = cluster.map_shared_rank(grp_slot, 0);
+    // (a streaming CTA on its own addresses its table directly: a mapped address takes the cluster's path even to itself)
+    const bool direct = STREAM && csize == 1;
+    DraftSmem* lsm = direct ? sm : cluster.map_shared_rank(sm, 0);
+    int* lrep = direct ? rep : cluster.map_shared_rank(rep, 0);
+    int* lcnt = direct ? cnt : cluster.map_shared_rank(cnt, 0);
+    int* llast = direct ? last : cluster.map_shared_rank(last, 0);
+    int* lgrp_slot = direct ? grp_slot : cluster.map_shared_rank(grp_slot, 0);
 
     // barrier over all CTAs of the sequence (a plain CTA barrier when there is only one: much cheaper)
     auto pass_sync = [&]() {
@@ -182,7 +195,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         if (tid == 0 && leader) atomicOr(P.status, SPEC_STATUS_CAPACITY);
         L = 0;
     }
-    if (P.stage_hist) {
+    if (!STREAM) {
         const int4* g4 = reinterpret_cast<const int4*>(h);
         int4* s4 = reinterpret_cast<int4*>(hist_s);
         const int n4 = (L + 3) >> 2;  // cap % 4 == 0 and L <= cap: the last vector stays inside the row
@@ -238,6 +251,12 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     bool any_q = false;
     for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + w);
 
+    const int4* h4 = reinterpret_cast<const int4*>(h);
+    const int n_vec_all = (max(n_scan, 0) + 3) >> 2;
+    const int v_chunk = (n_vec_all + csize - 1) / csize;  // this CTA's slice of the history
+    const int n_vec = min(n_vec_all, (crank + 1) * v_chunk);
+    int* wq = reinterpret_cast<int*>(smem_raw + P.queue_off) + warp * kMatchQueue;  // this warp's queue of matches
+
     int R = 1;
     bool gave_up = false;
     while (any_q && n_scan >= 1) {
@@ -257,69 +276,132 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                 }
             }
             pass_sync();  // the leader's table is ready
-            // scan: 128-bit loads, four per thread in flight; positions holding the last token are
-            // collected in a bit mask and handled one by one (they are rare)
-            const int4* h4 = reinterpret_cast<const int4*>(h);
-            const int n_vec_all = (n_scan + 3) >> 2;
-            const int v_chunk = (n_vec_all + csize - 1) / csize;  // this CTA's slice of the history
-            const int n_vec = min(n_vec_all, (crank + 1) * v_chunk);
+            // scan: positions holding the last token are collected in a bit mask and handled one by
+            // one (they are rare).  `hits` has bit 4u+c for component c of the lane's u-th vector.
             const bool need2 = P.q_min >= 2;  // every query has at least two tokens: test the second one in registers
+            // bits of one vector; `before` is the token left of the vector's first one
+            auto vec_hits = [&](const int4& v, int before, int xb) -> unsigned {
+                bool px = true, py = true, pz = true, pw = true;
+                if (need2) {
+                    px = before == t1;
+                    py = v.x == t1;
+                    pz = v.y == t1;
+                    pw = v.z == t1;
+                }
+                return (unsigned)(v.x == t0 && px && xb + 0 < n_scan) | (unsigned)(v.y == t0 && py && xb + 1 < n_scan) << 1 |
+                       (unsigned)(v.z == t0 && pz && xb + 2 < n_scan) << 2 | (unsigned)(v.w == t0 && pw && xb + 3 < n_scan) << 3;
+            };
+            // group the match at token index x (the continuation starts at x + 1)
+            auto handle_match = [&](int x) {
+                // length of the common suffix of hist[0..x] and the whole history, up to q_max
+                int m = 1;
+                if (P.q_max > 1 && x >= 1 && h[x - 1] == t1) {
+                    m = 2;
+                    if (P.q_max > 2 && x >= 2 && h[x - 2] == t2) {
+                        m = 3;
+                        if (P.q_max > 3 && x >= 3 && h[x - 3] == t3) m = 4;
+                    }
+                }
+                const int p = x + 1;
+                uint32_t hc = 0x9E3779B9u;
+                for (int t = 0; t < key_len; ++t) hc = fmix32(hc ^ (uint32_t)h[p + t]) + 0x7F4A7C15u;
+                for (int qi = 0; qi < P.n_q; ++qi) {
+                    const int q = P.qs[qi];
+                    if (m < q || L < q + w) continue;
+                    const uint32_t hq = fmix32(hc + (uint32_t)qi * 0x632BE5ABu);
+                    if (R > 1 && (int)(fmix32(hq ^ 0xA511E9B3u) % (uint32_t)R) != r) continue;
+                    insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, lrep, lcnt, llast, lgrp_slot, lsm);
+                }
+            };
+            // Matches are not grouped where they are found: a match costs a chain of dependent reads of
+            // the history (suffix, continuation, the group's representative), and a warp that stopped
+            // for each one would scan at the speed of that chain.  The warp queues the positions and
+            // groups a queue-full at a time, one match per lane, so the chains of 32 matches overlap.
+            int qn = 0;  // queued matches (the same in every lane)
+            auto flush_matches = [&]() {
+                __syncwarp();
+                for (int i = lane; i < qn; i += 32) handle_match(wq[i]);
+                __syncwarp();
+                qn = 0;
+            };
+            // v0 = the lane's first vector, its u-th vector is v0 + u * ustride
+            auto handle_hits = [&](unsigned hits, int v0, int ustride) {
+                if constexpr (!STREAM) {  // history in shared memory: a match costs no more than queueing it would
+                    while (hits) {
+                        const int bit = __ffs(hits) - 1;
+                        hits &= hits - 1;
+                        handle_match(((v0 + (bit >> 2) * ustride) << 2) + (bit & 3));
+                    }
+                    return;
+                } else {
+                if (!__any_sync(0xffffffffu, hits != 0u)) return;
+                const int nh = __popc(hits);
+                int incl = nh;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const int total = __shfl_sync(0xffffffffu, incl, 31);
+                if (total > kMatchQueue) {  // denser than the queue: group them in place
+                    while (hits) {
+                        const int bit = __ffs(hits) - 1;
+                        hits &= hits - 1;
+                        handle_match(((v0 + (bit >> 2) * ustride) << 2) + (bit & 3));
+                    }
+                    return;
+                }
+                if (qn + total > kMatchQueue) flush_matches();
+                int at = qn + incl - nh;
+                while (hits) {
+                    const int bit = __ffs(hits) - 1;
+                    hits &= hits - 1;
+                    wq[at++] = ((v0 + (bit >> 2) * ustride) << 2) + (bit & 3);
+                }
+                qn += total;
+                }
+            };
+            // 128-bit loads, four per thread in flight.  The common case (no match among the warp's
+            // 512 tokens) is decided by one comparison chain per vector and one vote; only then are
+            // the positions worked out.
             for (int vw = crank * v_chunk + (tid - lane); vw < n_vec; vw += 4 * nthr) {  // warp-uniform trip count
                 // too many groups for one pass: rescan with more passes
                 if (__any_sync(0xffffffffu, *((volatile int*)&lsm->overflow))) break;
                 const int v0 = vw + lane;
                 int4 vv[4];
+                int left[4];  // token before the vector: lane 0 asks for it together with the vectors
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int vi = v0 + u * nthr;
                     vv[u] = (vi < n_vec) ? h4[vi] : make_int4(-3, -3, -3, -3);
+                    if constexpr (STREAM) left[u] = (need2 && lane == 0 && vi > 0 && vi < n_vec) ? h[(vi << 2) - 1] : -5;
+                }
+                if constexpr (!STREAM) {
+                    if (need2) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int vi = v0 + u * nthr;
+                            left[u] = __shfl_up_sync(0xffffffffu, vv[u].w, 1);
+                            if (lane == 0) left[u] = (vi > 0 && vi < n_vec) ? h[(vi << 2) - 1] : -5;
+                        }
+                    }
+                } else if (need2) {  // token before each position: from this vector, or from the lane to the left
+                    bool some = false;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int up = __shfl_up_sync(0xffffffffu, vv[u].w, 1);
+                        if (lane != 0) left[u] = up;
+                        some = some || (vv[u].x == t0 && left[u] == t1) || (vv[u].y == t0 && vv[u].x == t1) ||
+                               (vv[u].z == t0 && vv[u].y == t1) || (vv[u].w == t0 && vv[u].z == t1);
+                    }
+                    if (!__any_sync(0xffffffffu, some)) continue;
                 }
                 unsigned hits = 0;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int vi = v0 + u * nthr;
-                    const int xb = vi << 2;
-                    bool px = true, py = true, pz = true, pw = true;
-                    if (need2) {  // token before each position: from this vector, or from the lane to the left
-                        int before = __shfl_up_sync(0xffffffffu, vv[u].w, 1);
-                        if (lane == 0) before = (vi > 0 && vi < n_vec) ? h[xb - 1] : -5;
-                        px = before == t1;
-                        py = vv[u].x == t1;
-                        pz = vv[u].y == t1;
-                        pw = vv[u].z == t1;
-                    }
-                    hits |= (unsigned)(vv[u].x == t0 && px && xb + 0 < n_scan) << (4 * u + 0);
-                    hits |= (unsigned)(vv[u].y == t0 && py && xb + 1 < n_scan) << (4 * u + 1);
-                    hits |= (unsigned)(vv[u].z == t0 && pz && xb + 2 < n_scan) << (4 * u + 2);
-                    hits |= (unsigned)(vv[u].w == t0 && pw && xb + 3 < n_scan) << (4 * u + 3);
-                }
-                while (hits) {
-                    const int bit = __ffs(hits) - 1;
-                    hits &= hits - 1;
-                    {
-                        const int x = ((v0 + (bit >> 2) * nthr) << 2) + (bit & 3);
-                        // length of the common suffix of hist[0..x] and the whole history, up to q_max
-                        int m = 1;
-                        if (P.q_max > 1 && x >= 1 && h[x - 1] == t1) {
-                            m = 2;
-                            if (P.q_max > 2 && x >= 2 && h[x - 2] == t2) {
-                                m = 3;
-                                if (P.q_max > 3 && x >= 3 && h[x - 3] == t3) m = 4;
-                            }
-                        }
-                        const int p = x + 1;
-                        uint32_t hc = 0x9E3779B9u;
-                        for (int t = 0; t < key_len; ++t) hc = fmix32(hc ^ (uint32_t)h[p + t]) + 0x7F4A7C15u;
-                        for (int qi = 0; qi < P.n_q; ++qi) {
-                            const int q = P.qs[qi];
-                            if (m < q || L < q + w) continue;
-                            const uint32_t hq = fmix32(hc + (uint32_t)qi * 0x632BE5ABu);
-                            if (R > 1 && (int)(fmix32(hq ^ 0xA511E9B3u) % (uint32_t)R) != r) continue;
-                            insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, lrep, lcnt, llast, lgrp_slot, lsm);
-                        }
-                    }
-                }
+                for (int u = 0; u < 4; ++u) hits |= vec_hits(vv[u], left[u], (v0 + u * nthr) << 2) << (4 * u);
+                handle_hits(hits, v0, nthr);
             }
+            if constexpr (STREAM) flush_matches();
             pass_sync();  // every CTA's matches are in the table
             const int ov = *((volatile int*)&lsm->overflow);
             pass_sync();  // every CTA has read the flag before the leader may reset it
@@ -563,9 +645,25 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.status = ctx->d_status;
     int slots = 1024;  // at most slots / 2 distinct continuations are grouped in one pass
     while (slots < cap / 2 && slots < 8192) slots <<= 1;
+    int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);
+    // A batch that fills the GPU more than once runs faster with two or three CTAs per SM (the scan of one
+    // overlaps the barriers and serial phases of another): half the threads, and half the table where few
+    // groups are expected (every query has two tokens or more, or the history is short).  Measured on
+    // S x L = 592 x 32768, 592 x 131072 and 2048 x 8192: 1.9x, 1.1x and 2.3x faster than the shape above.
+    if (S > ctx->num_sms && cap > 8192 && (P.q_min >= 2 || cap <= 16384)) {
+        threads = 512;
+        if (slots > 4096) slots = 4096;
+    }
+    // Tuning aid: NGRAM_SPEC_DRAFT_SHAPE="threads,slots" overrides the choice (values are clamped).
+    if (const char* ov = getenv("NGRAM_SPEC_DRAFT_SHAPE")) {
+        int t = 0, sl = 0;
+        if (sscanf(ov, "%d,%d", &t, &sl) == 2) {
+            if (t >= 128 && t <= 1024 && t % 32 == 0) threads = t;
+            if (sl >= 1024 && sl <= 8192 && (sl & (sl - 1)) == 0) slots = sl;
+        }
+    }
     P.slots = slots;
     P.max_groups = slots / 2;
-    const int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);
     // CTAs per sequence: one per 16K tokens of capacity, at most 8, and only while the batch alone
     // cannot fill the GPU (with many sequences one CTA each is the faster way to stream them)
     unsigned csize = 1;
@@ -575,16 +673,22 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     const size_t work_bytes = ((table_bytes > cand_bytes ? table_bytes : cand_bytes) + 15) & ~size_t(15);
     P.stage_hist = (csize == 1 && cap <= 8192) ? 1 : 0;
     P.hist_off = (int)(work_bytes / sizeof(int));
-    const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + work_bytes + (P.stage_hist ? (size_t)cap * sizeof(int32_t) : 0);
+    size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + work_bytes + (P.stage_hist ? (size_t)cap * sizeof(int32_t) : 0);
+    P.queue_off = (int)((smem + 15) & ~size_t(15));
+    smem = (size_t)P.queue_off + (size_t)(threads / 32) * kMatchQueue * sizeof(int);
     static bool attr_set[64] = {false};
     bool& attr_done = attr_set[ctx->device & 63];
     if (!attr_done) {
-        int rc = check_cuda(ctx, cudaFuncSetAttribute(draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024),
+        int rc = check_cuda(ctx, cudaFuncSetAttribute(draft_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024),
                             "draft: cudaFuncSetAttribute");
+        if (rc) return rc;
+        rc = check_cuda(ctx, cudaFuncSetAttribute(draft_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024),
+                        "draft: cudaFuncSetAttribute");
         if (rc) return rc;
         attr_done = true;
     }
-    cudaError_t e = launch_pdl_cluster(draft_kernel, dim3((unsigned)S * csize), dim3(threads), smem, st, csize, P);
+    cudaError_t e = launch_pdl_cluster(P.stage_hist ? draft_kernel<false> : draft_kernel<true>, dim3((unsigned)S * csize),
+                                       dim3(threads), smem, st, csize, P);
     ctx->launches += 1;
     return check_cuda(ctx, e, "draft_context_ngrams launch");
 }
