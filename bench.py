@@ -637,7 +637,7 @@ def main():
 
 # DRAM bytes per verify launch from the ncu captures summarised under profiles/ (None = not captured
 # for the current kernel).
-TRAFFIC = {"C2": 266.1e6, "C3": 1.658e9}
+TRAFFIC = {"C2": 267.0e6, "C3": 1.688e9}
 
 
 def run_reference(args, c, cfg):

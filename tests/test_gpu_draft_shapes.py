@@ -54,3 +54,30 @@ def test_random_draft_problem(ctx, case):
     for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
         assert np.array_equal(a.cpu().numpy(), b), name
     assert ctx.get_status() == 0
+
+
+@pytest.mark.parametrize("alpha,qs,Lmax", [(3, [1], 9000), (40, [2, 1], 12000), (6, [3, 2], 17000), (V, [2], 9500),
+                                           (2, [4, 3], 8400), (6, [1], 16000)])
+def test_batch_of_unstaged_histories(ctx, alpha, qs, Lmax):
+    """More sequences than SMs, histories too long to stage in shared memory: the batch launch shape
+    (several CTAs per SM, smaller table) and the queued grouping of matches, from a few matches per
+    warp iteration (queue filled and flushed in mid-scan) to more than a queue holds (grouped in place);
+    the last case has more distinct continuations than the smaller table groups in one pass."""
+    g = np.random.default_rng(31000 + alpha + Lmax)
+    S, B, w, topk, k_tab = 160, 12, 5, 6, 4
+    cap = Lmax + 8
+    lens = np.array([Lmax if s % 7 == 0 else int(g.integers(Lmax // 2, Lmax + 1)) for s in range(S)], np.int32)
+    hist = np.full((S, cap), -1, np.int32)
+    for s in range(S):
+        h = g.integers(0, alpha, lens[s])
+        for _ in range(int(lens[s]) // 200):
+            a, b, n = int(g.integers(0, lens[s] - 20)), int(g.integers(0, lens[s] - 20)), int(g.integers(4, 20))
+            h[b:b + n] = h[a:a + n]
+        hist[s, :lens[s]] = h
+    T = np.stack([g.permutation(V)[:k_tab] for _ in range(V)]).astype(np.int32)
+    ctx.set_model_table(dev_i32(T), None)
+    want = oracle.draft_batch(hist, lens, qs, topk, B, w, 3, T)
+    got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, 3)
+    for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
+        assert np.array_equal(a.cpu().numpy(), b), name
+    assert ctx.get_status() == 0
