@@ -15,7 +15,8 @@
 // the scan, the key comparisons and the candidate rows then never wait for global memory again,
 // which is what the latency of a single short sequence is made of.
 //
-// The scan itself only looks for matches: per 128-bit vector one comparison chain, per warp iteration
+// On the throughput path (one CTA per sequence, history read from global memory) the scan itself only
+// looks for matches: per 128-bit vector one comparison chain, per warp iteration
 // (512 tokens) one vote.  Where a match turns up its position goes into a per-warp queue, and a
 // queue-full of matches is grouped at once, one per lane, so that the dependent reads each match
 // needs (suffix, continuation, the group's representative) overlap instead of stalling the scan.
@@ -137,9 +138,11 @@ __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int 
     sm->overflow = 1;
 }
 
-// STREAM = false: the history was staged in shared memory (one CTA, short history; the latency of this
-// instantiation is a step's drafting latency, so it carries nothing it does not execute).
-// STREAM = true: the history is read from global memory, by one CTA or by a cluster.
+// STREAM = false: the latency path - a short history staged in shared memory (one CTA; a decode step's
+// drafting latency, so this instantiation carries nothing it does not execute), or a long history split
+// over a cluster (few sequences: matches are grouped where they are found, which also notices a full
+// table at once and cuts a void pass short).
+// STREAM = true: the throughput path - one CTA per sequence reading its history from global memory.
 template <bool STREAM>
 __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -155,8 +158,8 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     cg::cluster_group cluster = cg::this_cluster();
     const int csize = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
     const bool leader = crank == 0;
-    // (a streaming CTA on its own addresses its table directly: a mapped address takes the cluster's path even to itself)
-    const bool direct = STREAM && csize == 1;
+    // (the throughput path addresses its table directly: a mapped address takes the cluster's path even to itself)
+    const bool direct = STREAM;
     DraftSmem* lsm = direct ? sm : cluster.map_shared_rank(sm, 0);
     int* lrep = direct ? rep : cluster.map_shared_rank(rep, 0);
     int* lcnt = direct ? cnt : cluster.map_shared_rank(cnt, 0);
@@ -195,7 +198,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         if (tid == 0 && leader) atomicOr(P.status, SPEC_STATUS_CAPACITY);
         L = 0;
     }
-    if (!STREAM) {
+    if (P.stage_hist) {
         const int4* g4 = reinterpret_cast<const int4*>(h);
         int4* s4 = reinterpret_cast<int4*>(hist_s);
         const int n4 = (L + 3) >> 2;  // cap % 4 == 0 and L <= cap: the last vector stays inside the row
@@ -326,7 +329,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             };
             // v0 = the lane's first vector, its u-th vector is v0 + u * ustride
             auto handle_hits = [&](unsigned hits, int v0, int ustride) {
-                if constexpr (!STREAM) {  // history in shared memory: a match costs no more than queueing it would
+                if constexpr (!STREAM) {
                     while (hits) {
                         const int bit = __ffs(hits) - 1;
                         hits &= hits - 1;
@@ -687,7 +690,7 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
         if (rc) return rc;
         attr_done = true;
     }
-    cudaError_t e = launch_pdl_cluster(P.stage_hist ? draft_kernel<false> : draft_kernel<true>, dim3((unsigned)S * csize),
+    cudaError_t e = launch_pdl_cluster((P.stage_hist || csize > 1) ? draft_kernel<false> : draft_kernel<true>, dim3((unsigned)S * csize),
                                        dim3(threads), smem, st, csize, P);
     ctx->launches += 1;
     return check_cuda(ctx, e, "draft_context_ngrams launch");
