@@ -56,9 +56,10 @@ def test_random_draft_problem(ctx, case):
     assert ctx.get_status() == 0
 
 
-@pytest.mark.parametrize("alpha,qs,Lmax", [(3, [1], 9000), (40, [2, 1], 12000), (6, [3, 2], 17000), (V, [2], 9500),
-                                           (2, [4, 3], 8400), (6, [1], 16000)])
-def test_batch_of_unstaged_histories(ctx, alpha, qs, Lmax):
+@pytest.mark.parametrize("alpha,qs,Lmax,flags", [(3, [1], 9000, 3), (40, [2, 1], 12000, 7), (6, [3, 2], 17000, 3),
+                                                 (V, [2], 9500, 1), (2, [4, 3], 8400, 5), (6, [1], 16000, 3),
+                                                 (40, [1, 2], 10000, 2)])
+def test_batch_of_unstaged_histories(ctx, alpha, qs, Lmax, flags):
     """More sequences than SMs, histories too long to stage in shared memory: the batch launch shape
     (several CTAs per SM, smaller table) and the queued grouping of matches, from a few matches per
     warp iteration (queue filled and flushed in mid-scan) to more than a queue holds (grouped in place);
@@ -76,8 +77,8 @@ def test_batch_of_unstaged_histories(ctx, alpha, qs, Lmax):
         hist[s, :lens[s]] = h
     T = np.stack([g.permutation(V)[:k_tab] for _ in range(V)]).astype(np.int32)
     ctx.set_model_table(dev_i32(T), None)
-    want = oracle.draft_batch(hist, lens, qs, topk, B, w, 3, T)
-    got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, 3)
+    want = oracle.draft_batch(hist, lens, qs, topk, B, w, flags, T)
+    got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, flags)
     for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
         assert np.array_equal(a.cpu().numpy(), b), name
     assert ctx.get_status() == 0
