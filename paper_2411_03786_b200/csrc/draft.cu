@@ -677,8 +677,9 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.stage_hist = (csize == 1 && cap <= 8192) ? 1 : 0;
     P.hist_off = (int)(work_bytes / sizeof(int));
     size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + work_bytes + (P.stage_hist ? (size_t)cap * sizeof(int32_t) : 0);
+    const bool throughput = !P.stage_hist && csize == 1;  // which instantiation runs (see draft_kernel)
     P.queue_off = (int)((smem + 15) & ~size_t(15));
-    smem = (size_t)P.queue_off + (size_t)(threads / 32) * kMatchQueue * sizeof(int);
+    if (throughput) smem = (size_t)P.queue_off + (size_t)(threads / 32) * kMatchQueue * sizeof(int);  // per-warp match queues
     static bool attr_set[64] = {false};
     bool& attr_done = attr_set[ctx->device & 63];
     if (!attr_done) {
@@ -690,7 +691,7 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
         if (rc) return rc;
         attr_done = true;
     }
-    cudaError_t e = launch_pdl_cluster((P.stage_hist || csize > 1) ? draft_kernel<false> : draft_kernel<true>, dim3((unsigned)S * csize),
+    cudaError_t e = launch_pdl_cluster(throughput ? draft_kernel<true> : draft_kernel<false>, dim3((unsigned)S * csize),
                                        dim3(threads), smem, st, csize, P);
     ctx->launches += 1;
     return check_cuda(ctx, e, "draft_context_ngrams launch");
