@@ -97,8 +97,11 @@ def extend_table(T, w: int) -> np.ndarray:
     return ext
 
 
-def draft_batch(hist, lens, qs, topk: int, B: int, w: int, flags: int = FLAG_DEDUP | FLAG_MODEL_FILL, T=None):
-    """Section 4.3 mixed strategy for S sequences.  Returns drafts[S,B,w], n_drafts[S], src[S,B], counts[S,B]."""
+def draft_batch(hist, lens, qs, topk: int, B: int, w: int, flags: int = FLAG_DEDUP | FLAG_MODEL_FILL, T=None, V: int | None = None):
+    """Section 4.3 mixed strategy for S sequences.  Returns drafts[S,B,w], n_drafts[S], src[S,B], counts[S,B].
+
+    ``V`` (default: the table's row count, else unknown) is the vocabulary size: when known, a context
+    row holding a token outside [0, V) is passed over."""
     hist = _i32(hist)
     lens = _i32(lens)
     S, cap = hist.shape
@@ -109,9 +112,10 @@ def draft_batch(hist, lens, qs, topk: int, B: int, w: int, flags: int = FLAG_DED
     counts = np.empty((S, B), dtype=np.int32)
     if T is not None:
         T = _i32(T)
-        V, k_tab = T.shape
+        k_tab = T.shape[1]
+        V = T.shape[0] if V is None else V
     else:
-        V, k_tab = 0, 0
+        V, k_tab = (0 if V is None else V), 0
     lib().oracle_draft_batch(_p(hist, C.c_int32), _p(lens, C.c_int32), S, cap, qs_arr, len(qs), int(topk), int(B),
                              int(w), int(flags), _p(T, C.c_int32), V, k_tab,
                              _p(drafts, C.c_int32), _p(nd, C.c_int32), _p(src, C.c_int32), _p(counts, C.c_int32))

@@ -171,6 +171,13 @@ int oracle_draft_sequence(const int32_t* hist, int L, const int* qs, int n_q, in
         int m = oracle_context_draft_keyed(hist, L, qs[qi], w, (flags & 4) ? 1 : w, topk, cand, cnt, NULL);
         for (int r = 0; r < m && n < ctx_cap; ++r) {
             int dup = 0;
+            /* The paper's tokens are elements of the vocabulary by definition (Section 2).  When the
+             * vocabulary size is known (V > 0), a ranked continuation that carries a token outside
+             * [0, V) -- a corrupt history -- is passed over: it takes no draft row. */
+            int in_range = 1;
+            for (int t = 0; t < w && V > 0; ++t)
+                if (cand[r * w + t] < 0 || cand[r * w + t] >= V) in_range = 0;
+            if (!in_range) continue;
             if (dedup)
                 for (int b = 0; b < n && !dup; ++b)
                     if (memcmp(drafts + b * w, cand + r * w, sizeof(int32_t) * (size_t)w) == 0) dup = 1;
@@ -201,7 +208,6 @@ int oracle_draft_sequence(const int32_t* hist, int L, const int* qs, int n_q, in
         }
     }
     free(cand); free(cnt);
-    (void)V;
     return n;
 }
 

@@ -190,6 +190,33 @@ def test_rows_reserved_for_the_model_cap_the_context_rows():
     assert src[0, :nd[0]].tolist() == [0] * int(nd[0])                        # everything reserved: model rows only
 
 
+def test_context_row_with_a_token_outside_the_vocabulary_is_passed_over():
+    # after token 1: (2, 9) at 1 and (3, 1) at 4, once each => ranked by recency (3, 1), (2, 9); with V = 5 the
+    # token 9 is not a vocabulary entry, so that row takes no draft row (and the rows behind it move up)
+    T = np.array([[1, 2], [2, 0], [0, 1], [4, 0], [0, 3]], np.int32)
+    hist = np.array([[1, 2, 9, 1, 3, 1, -1, -1]], np.int32)
+    lens = np.array([6], np.int32)
+    d, nd, src, cnt = oracle.draft_batch(hist, lens, [1], 4, 4, 2, 1, None)          # vocabulary unknown: both rows
+    assert nd[0] == 2 and d[0, :2].tolist() == [[3, 1], [2, 9]]
+    d, nd, src, cnt = oracle.draft_batch(hist, lens, [1], 4, 4, 2, 1, None, V=5)
+    assert nd[0] == 1 and d[0].tolist() == [[3, 1], [-1, -1], [-1, -1], [-1, -1]] and src[0].tolist() == [1, -1, -1, -1]
+    d, nd, src, cnt = oracle.draft_batch(hist, lens, [1], 4, 4, 2, 3, T)              # V from the table; model rows follow
+    assert nd[0] == 3 and d[0, :3].tolist() == [[3, 1], [2, 0], [0, 1]] and src[0, :3].tolist() == [1, 0, 0]
+    # brute force on random histories over {0..5} with V = 4: rows holding 4 or 5 vanish, the order of the rest is kept
+    g = np.random.default_rng(17)
+    for _ in range(100):
+        L = int(g.integers(4, 50))
+        h = g.integers(0, 6, L).astype(np.int32)
+        h[-1] = g.integers(0, 4)
+        w, topk = int(g.integers(1, 4)), int(g.integers(1, 6))
+        h2 = np.full((1, (L + 3) // 4 * 4 + 4), -1, np.int32)
+        h2[0, :L] = h
+        rows, _, _ = brute_mix(h, [2, 1], topk, 64, w, 1, None)
+        keep = [r for r in rows if all(0 <= t < 4 for t in r)]
+        d, nd, _, _ = oracle.draft_batch(h2, np.array([L], np.int32), [2, 1], topk, 64, w, 1, None, V=4)
+        assert d[0, :nd[0]].tolist() == keep
+
+
 def test_ablation_counters_hand_example():
     # three sequences, B = 3, w = 2
     src = np.array([[1, 1, 0], [2, 0, -1], [0, 0, 0]], np.int32)
