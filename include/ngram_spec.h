@@ -33,6 +33,10 @@
  *     for every buffer; other work enqueued before or after behaves as with ordinary launches.
  *   - The GPU must be compute capability 10.0 (sm_100a).  There is no CPU fallback: every entry
  *     point fails with SPEC_ERR_CUDA when no such device is usable.
+ *   - Host threads: a context is used by one host thread at a time (it caches tensor maps and keeps
+ *     its error text); different contexts may be driven from different threads at the same time --
+ *     the library's process-wide caches are locked, and spec_last_error(NULL) is per thread.  The
+ *     library reads no environment variables.
  */
 #ifndef NGRAM_SPEC_H_
 #define NGRAM_SPEC_H_
@@ -55,7 +59,7 @@ enum {
 
 /* bits of the device status word */
 enum {
-    SPEC_STATUS_TOKEN_RANGE = 1, /* a token outside [0, V) was met; the affected row was dropped */
+    SPEC_STATUS_TOKEN_RANGE = 1, /* a draft row (context or model) held a token outside [0, V): the row was dropped */
     SPEC_STATUS_CAPACITY = 2,    /* len > cap, or a commit did not fit: that sequence was skipped */
     SPEC_STATUS_TIMEOUT = 4,     /* a bounded device-side wait expired; results of that call are invalid */
     SPEC_STATUS_GROUPS = 8       /* more distinct continuations than the drafter can group exactly */
@@ -107,6 +111,18 @@ int build_model_ngram_tables(spec_ctx* ctx, const void* d_rows, int k_tab, int w
                              float* d_tab_val, int32_t* d_ext, void* stream);
 
 /*
+ * The same table built in slices, for several GPUs (rows of the table are independent: Section 4.1
+ * computes p_M(.|x) one token x at a time).  Writes rows [row_begin, row_begin + row_count) of d_tab_idx
+ * (and d_tab_val), which are the WHOLE [V, k_tab] arrays; d_rows, if given, is the whole [V, d] matrix.
+ * Each rank builds its slice, the slices are exchanged (an all-gather of row_count * k_tab int32 per
+ * rank), and spec_extend_model_table then derives the w-token extension from the complete table and
+ * adopts both for draft_context_ngrams.  Nothing is adopted by build_model_ngram_table_rows itself.
+ */
+int build_model_ngram_table_rows(spec_ctx* ctx, const void* d_rows, int row_begin, int row_count, int k_tab,
+                                 int32_t* d_tab_idx, float* d_tab_val, void* stream);
+int spec_extend_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, int w_ext, int32_t* d_ext, void* stream);
+
+/*
  * Model unigram (Section 4.1 "Unigram").  d(x) = || u_x - ubar ||_V: u_x is row x of the unembedding,
  * ubar the mean row, and the norm is induced by <a, b>_V = sum_y (a . v_y)(b . v_y) over the rows v_y
  * of the embedding.  p(x) is proportional to exp(-d(x)), so the top-k unigram tokens are the k with the
@@ -149,6 +165,7 @@ int draft_context_ngrams(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_
  * b of sequence s (column 0 = the last context token).
  *   d_hidden   [M, d] bfloat16.      d_max  [M] float32 out or NULL (the winning logit).
  * Uses the context's merge keys as scratch: calls on one context must not overlap on the GPU.
+ * If a bounded device-side wait expires (SPEC_STATUS_TIMEOUT), every row of d_argmax is -1.
  */
 int verify_lmhead_argmax(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max,
                          void* stream);
@@ -252,17 +269,32 @@ int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits,
  *
  *   - M may not exceed SPEC_NOALLOC_MAX_ROWS; a larger M is rejected with SPEC_ERR_ARG.  The array
  *     (about 33 KB) is held by every GPU that loads the library, until the process exits.
- *   - It calls no cudaMalloc / cudaFree and no allocating routine; it enqueues three small memsets
- *     and one kernel on `stream`.
+ *   - It calls no cudaMalloc / cudaFree and no routine that allocates device memory; it enqueues
+ *     three small memsets and one kernel on `stream`.  ("Allocates nothing" is about device memory:
+ *     the first call for a new block height may add an entry to a small host-side table.)
  *   - The first call on each device looks up the array's device address and the driver's
- *     tensor-map encoder; make that first call before any stream capture begins.
+ *     tensor-map encoder; make that first call before any stream capture begins.  The set-up is
+ *     locked, so two host threads may both make "the first call".
  *   - All calls share the one array and it keeps the previous call's contents, so the call clears
  *     what it needs first.  Two calls whose GPU work overlaps (different streams, or different
  *     threads) race on it: serialise them.
- *   - d_argmax is pre-set to -1; if a bounded device-side wait ever expired the rows stay -1.
+ *   - If a bounded device-side wait expires inside the kernel, every row of d_argmax is -1 (and
+ *     d_max is -inf): the call has no status word a caller could read, so -1 is its error signal.
  */
 int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d, const void* d_hidden, int M,
                                  int32_t* d_argmax, float* d_max, int device, void* stream);
+
+/*
+ * Test aid for the bounded device-side waits.  Every wait inside the kernels (on an mbarrier that a
+ * copy or the tensor cores complete) gives up after a time limit, sets SPEC_STATUS_TIMEOUT and lets the
+ * kernel return, so that a lost completion cannot hang the GPU.  This call runs a one-thread kernel that
+ * waits, with that same routine and a limit of limit_ns (at most one second), on a barrier nobody arrives
+ * at: afterwards spec_get_status reports SPEC_STATUS_TIMEOUT and the context is usable as before.  With
+ * mark_verify_incomplete != 0 the kernel also registers itself the way a contraction CTA that gave up
+ * does, so the NEXT verify_lmhead_argmax on this context reports every row as -1 (d_max = -inf, exported
+ * keys = the smallest key) instead of a partial arg max; the verification after that is normal again.
+ */
+int spec_debug_expire_wait(spec_ctx* ctx, unsigned long long limit_ns, int mark_verify_incomplete, void* stream);
 
 /* Number of kernels the library has launched for this context since spec_init. */
 long long spec_launch_count(spec_ctx* ctx);

@@ -67,6 +67,9 @@ def load_library(build: bool = True) -> C.CDLL:
     lib.spec_set_head_fp8.argtypes = [vp, vp, fp]
     lib.verify_lmhead_argmax_fp8.argtypes = [vp, vp, C.c_int, vp, fp, i32p, fp, vp]
     lib.verify_lmhead_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, i32p, fp, C.c_int, vp]
+    lib.build_model_ngram_table_rows.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, i32p, fp, vp]
+    lib.spec_extend_model_table.argtypes = [vp, i32p, C.c_int, C.c_int, i32p, vp]
+    lib.spec_debug_expire_wait.argtypes = [vp, C.c_ulonglong, C.c_int, vp]
     lib.spec_launch_count.argtypes = [vp]
     lib.spec_launch_count.restype = C.c_longlong
     _lib = lib
@@ -139,6 +142,28 @@ class SpecContext:
                                                        _ptr(val), _ptr(ext), _stream()), "build_model_ngram_tables")
         self._keep_table = (tab, ext, rows)
         return tab, val, ext
+
+    def build_model_ngram_table_rows(self, k_tab: int, row_begin: int, row_count: int, tab: torch.Tensor,
+                                     val: torch.Tensor | None = None, rows: torch.Tensor | None = None):
+        """Writes rows ``[row_begin, row_begin + row_count)`` of the whole ``tab[V, k_tab]`` (one rank's slice)."""
+        assert tuple(tab.shape) == (self.V, k_tab)
+        self._check(self._lib.build_model_ngram_table_rows(self._h, _ptr(rows, torch.bfloat16), int(row_begin), int(row_count),
+                                                           k_tab, _ptr(tab, torch.int32), _ptr(val, torch.float32), _stream()),
+                    "build_model_ngram_table_rows")
+        return tab
+
+    def extend_model_table(self, tab: torch.Tensor, w_ext: int):
+        """Extension ``ext[V, k_tab, w_ext]`` of a complete table; adopts both for drafting."""
+        k_tab = int(tab.shape[1])
+        ext = torch.empty((self.V, k_tab, w_ext), dtype=torch.int32, device=tab.device)
+        self._check(self._lib.spec_extend_model_table(self._h, _ptr(tab, torch.int32), k_tab, int(w_ext), _ptr(ext), _stream()),
+                    "spec_extend_model_table")
+        self._keep_table = (tab, ext, None)
+        return ext
+
+    def debug_expire_wait(self, limit_ns: int = 20000, mark_verify_incomplete: bool = False):
+        self._check(self._lib.spec_debug_expire_wait(self._h, int(limit_ns), int(mark_verify_incomplete), _stream()),
+                    "spec_debug_expire_wait")
 
     def build_model_unigram(self, k_uni: int):
         """Returns ``(ids[k_uni] by ascending distance, dist2[V])``."""

@@ -2,14 +2,22 @@
 #include <stdarg.h>
 #include <string.h>
 
+#include <mutex>
+
 #include <cuda_bf16.h>
 
 #include "accept.cuh"
 #include "common.cuh"
 
-static char g_err[256] = "";
+// Error text of calls that have no context to keep it in: one buffer per host thread.
+static thread_local char g_err[256] = "";
 
 namespace ngs {
+
+std::mutex& host_mutex() {
+    static std::mutex m;
+    return m;
+}
 
 int fail(spec_ctx* ctx, int code, const char* fmt, ...) {
     char buf[256];
@@ -139,10 +147,10 @@ int spec_init(spec_ctx** out, const void* d_embed, const void* d_unembed, int dt
         if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_status, sizeof(int)), "cudaMalloc(status)"))) break;
         if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_keys, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS),
                              "cudaMalloc(keys)"))) break;
-        if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_ticket, sizeof(unsigned int)), "cudaMalloc(ticket)"))) break;
+        if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_ticket, 2 * sizeof(unsigned int)), "cudaMalloc(ticket)"))) break;
         cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st);
         cudaMemsetAsync(ctx->d_keys, 0, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS, st);
-        cudaMemsetAsync(ctx->d_ticket, 0, sizeof(unsigned int), st);
+        cudaMemsetAsync(ctx->d_ticket, 0, 2 * sizeof(unsigned int), st);
         if ((rc = make_w_maps(ctx, &ctx->tm_w, ctx->unembed, 2))) {
             strncpy(g_err, ctx->err, 255);
             break;
@@ -207,8 +215,35 @@ int build_model_ngram_tables(spec_ctx* ctx, const void* d_rows, int k_tab, int w
     if ((d_rows && !aligned16(d_rows)) || !aligned16(d_tab_idx))
         return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_tables: pointers must be 16-byte aligned");
     cudaSetDevice(ctx->device);
-    int rc = launch_table(ctx, d_rows ? d_rows : ctx->embed, k_tab, w_ext, d_tab_idx, d_tab_val, d_ext,
-                          (cudaStream_t)stream);
+    int rc = launch_table(ctx, d_rows ? d_rows : ctx->embed, ctx->V, k_tab, d_tab_idx, d_tab_val, (cudaStream_t)stream);
+    if (rc) return rc;
+    if (d_ext && (rc = launch_extend_table(ctx, d_tab_idx, k_tab, w_ext, d_ext, (cudaStream_t)stream))) return rc;
+    return spec_set_model_table(ctx, d_tab_idx, k_tab, d_ext, w_ext);
+}
+
+int build_model_ngram_table_rows(spec_ctx* ctx, const void* d_rows, int row_begin, int row_count, int k_tab,
+                                 int32_t* d_tab_idx, float* d_tab_val, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "build_model_ngram_table_rows: ctx is NULL");
+    if (!d_tab_idx) return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_table_rows: d_tab_idx is NULL");
+    if (k_tab < 1 || k_tab > kMaxKTab || k_tab > ctx->V)
+        return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_table_rows: k_tab must be in [1, min(%d, V)]", kMaxKTab);
+    if (row_begin < 0 || row_count < 0 || (long long)row_begin + row_count > ctx->V)
+        return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_table_rows: rows [%d, %d + %d) are not inside [0, V)", row_begin, row_begin, row_count);
+    if (d_rows && !aligned16(d_rows)) return fail(ctx, SPEC_ERR_ARG, "build_model_ngram_table_rows: d_rows must be 16-byte aligned");
+    if (row_count == 0) return SPEC_OK;
+    cudaSetDevice(ctx->device);
+    const char* a = (const char*)(d_rows ? d_rows : ctx->embed) + (size_t)row_begin * ctx->d * 2;  // d % 8 == 0: stays 16-byte aligned
+    return launch_table(ctx, a, row_count, k_tab, d_tab_idx + (size_t)row_begin * k_tab,
+                        d_tab_val ? d_tab_val + (size_t)row_begin * k_tab : nullptr, (cudaStream_t)stream);
+}
+
+int spec_extend_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, int w_ext, int32_t* d_ext, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_extend_model_table: ctx is NULL");
+    if (!d_tab_idx || !d_ext) return fail(ctx, SPEC_ERR_ARG, "spec_extend_model_table: NULL pointer");
+    if (k_tab < 1 || k_tab > kMaxKTab) return fail(ctx, SPEC_ERR_ARG, "spec_extend_model_table: k_tab must be in [1, %d]", kMaxKTab);
+    if (w_ext < 1 || w_ext > kMaxW) return fail(ctx, SPEC_ERR_ARG, "spec_extend_model_table: w_ext must be in [1, %d]", kMaxW);
+    cudaSetDevice(ctx->device);
+    int rc = launch_extend_table(ctx, d_tab_idx, k_tab, w_ext, d_ext, (cudaStream_t)stream);
     if (rc) return rc;
     return spec_set_model_table(ctx, d_tab_idx, k_tab, d_ext, w_ext);
 }
@@ -342,6 +377,7 @@ int spec_set_head_fp8(spec_ctx* ctx, const uint8_t* d_wq, const float* d_wscale)
     ctx->wq = d_wq;
     ctx->wscale = d_wscale;
     ctx->tm_q_ready = false;
+    ctx->wq_fresh = true;
     return SPEC_OK;
 }
 
@@ -369,6 +405,13 @@ int spec_debug_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits,
     if (m == 0) return SPEC_OK;
     cudaSetDevice(ctx->device);
     return launch_logits(ctx, d_rows, m, d_logits, (cudaStream_t)stream);
+}
+
+int spec_debug_expire_wait(spec_ctx* ctx, unsigned long long limit_ns, int mark_verify_incomplete, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_debug_expire_wait: ctx is NULL");
+    if (limit_ns > 1000000000ull) return fail(ctx, SPEC_ERR_ARG, "spec_debug_expire_wait: the limit may not exceed one second");
+    cudaSetDevice(ctx->device);
+    return launch_wait_probe(ctx, limit_ns, mark_verify_incomplete ? 1 : 0, (cudaStream_t)stream);
 }
 
 }  // extern "C"

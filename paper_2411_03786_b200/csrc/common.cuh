@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stdio.h>
 
+#include <mutex>
 #include <utility>
 
 #include "../../include/ngram_spec.h"
@@ -40,7 +41,7 @@ struct spec_ctx {
     int* d_status = nullptr;        // device status word
     // verify merge scratch: one packed (value, ~index) key per row + completion ticket
     unsigned long long* d_keys = nullptr;
-    unsigned int* d_ticket = nullptr;
+    unsigned int* d_ticket = nullptr;  // [0] CTAs finished, [1] CTAs that gave up on a bounded wait
     // table-build scratch: partial top-k lists per vocabulary chunk
     float* d_part_val = nullptr;
     int32_t* d_part_idx = nullptr;
@@ -61,6 +62,7 @@ struct spec_ctx {
     const float* wscale = nullptr;
     ngs::WMaps tm_q;
     bool tm_q_ready = false;
+    bool wq_fresh = false;  // the 8-bit head was set since the last verification over it
     // tensor maps of the most recent A operands (hidden states), so a decode loop that verifies from the
     // same buffer every step does not re-encode the map on every call
     struct AMap {
@@ -125,6 +127,10 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
 
+// Guards the process-wide host-side caches (launch shapes, per-device kernel attributes): contexts on
+// different host threads may call into the library at the same time.
+std::mutex& host_mutex();
+
 int fail(spec_ctx* ctx, int code, const char* fmt, ...);
 int check_cuda(spec_ctx* ctx, cudaError_t e, const char* what);
 bool aligned16(const void* p);
@@ -146,10 +152,11 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
                       cudaStream_t st);
 int launch_quantize_rows(spec_ctx* ctx, const void* d_rows, int n_rows, uint8_t* d_codes, float* d_scale, cudaStream_t st);
 int launch_unpack_keys(const long long* d_keys, int M, int V_total, int32_t* d_argmax, float* d_max, cudaStream_t st);
-int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
-                 int32_t* d_ext, cudaStream_t st);
+int launch_table(spec_ctx* ctx, const void* d_rows, int n_rows, int k_tab, int32_t* d_tab_idx, float* d_tab_val, cudaStream_t st);
+int launch_extend_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, int w_ext, int32_t* d_ext, cudaStream_t st);
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st);
 int launch_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2, cudaStream_t st);
+int launch_wait_probe(spec_ctx* ctx, unsigned long long limit_ns, int mark_incomplete, cudaStream_t st);
 // draft.cu / accept.cu
 int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
                  int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,

@@ -531,9 +531,21 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
             tok = keep ? sm->chain[r][t] : -1;
         } else {
             const unsigned long long key = sm->run_key[li][r];
-            tok = h[(int)(uint32_t)key + t];
+            const int start = (int)(uint32_t)key;
+            tok = h[start + t];
             src = P.qs[li];
             count = (int)(key >> 32);
+            if (t == 0) {
+                // a context row that carries a token outside the vocabulary (a corrupt history) is dropped, like
+                // a model row whose chain left it: the caller indexes its embedding table with these tokens
+                bool in_range = true;
+                for (int u = 0; u < w; ++u) {
+                    const int tk = h[start + u];
+                    in_range = in_range && tk >= 0 && tk < P.V;
+                }
+                keep = in_range ? 1 : 0;
+                if (!in_range) atomicOr(P.status, SPEC_STATUS_TOKEN_RANGE);
+            }
         }
         cand[i] = tok;
         if (t == 0) {
@@ -544,6 +556,7 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
         }
     }
     __syncthreads();
+
     // Rows reserved for the model strategy: the context strategies together take at most B - reserve.
     const int reserve = min(P.B, (P.flags >> 8) & 0xFF);
     const int n_ctx = sm->cand_off[P.n_q];
@@ -657,7 +670,8 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
         threads = 512;
         if (slots > 4096) slots = 4096;
     }
-    // Tuning aid: NGRAM_SPEC_DRAFT_SHAPE="threads,slots" overrides the choice (values are clamped).
+#ifdef NGRAM_SPEC_TUNING
+    // Tuning builds only: NGRAM_SPEC_DRAFT_SHAPE="threads,slots" overrides the choice (values are clamped).
     if (const char* ov = getenv("NGRAM_SPEC_DRAFT_SHAPE")) {
         int t = 0, sl = 0;
         if (sscanf(ov, "%d,%d", &t, &sl) == 2) {
@@ -665,6 +679,7 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
             if (sl >= 1024 && sl <= 8192 && (sl & (sl - 1)) == 0) slots = sl;
         }
     }
+#endif
     P.slots = slots;
     P.max_groups = slots / 2;
     // CTAs per sequence: one per 16K tokens of capacity, at most 8, and only while the batch alone
@@ -681,6 +696,7 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.queue_off = (int)((smem + 15) & ~size_t(15));
     if (throughput) smem = (size_t)P.queue_off + (size_t)(threads / 32) * kMatchQueue * sizeof(int);  // per-warp match queues
     static bool attr_set[64] = {false};
+    std::unique_lock<std::mutex> lock(host_mutex());
     bool& attr_done = attr_set[ctx->device & 63];
     if (!attr_done) {
         int rc = check_cuda(ctx, cudaFuncSetAttribute(draft_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024),
@@ -691,6 +707,7 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
         if (rc) return rc;
         attr_done = true;
     }
+    lock.unlock();
     cudaError_t e = launch_pdl_cluster(throughput ? draft_kernel<true> : draft_kernel<false>, dim3((unsigned)S * csize),
                                        dim3(threads), smem, st, csize, P);
     ctx->launches += 1;

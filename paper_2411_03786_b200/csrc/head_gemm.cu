@@ -50,7 +50,7 @@ constexpr int SMEM_MISC = 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int ACC_COLS = 256;                           // TMEM columns per accumulator stage
 constexpr int TMEM_COLS = 512;
 constexpr int GEMM_THREADS = 192;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // default limit of every device-side wait
 
 enum { MODE_ARGMAX = 0, MODE_TOPK = 1, MODE_STORE = 2, MODE_SUMSQ = 3, MODE_ARGMAX_Q8 = 4 };
 
@@ -88,6 +88,8 @@ struct GemmParams {
     int idx_offset;       // first token id of this shard
     const float* col_scale;  // 8-bit mode: scale of each row of W (= column of the product)
     const float* row_scale;  // 8-bit mode: scale of each row of A (only the reported maximum needs it)
+    unsigned long long wait_limit_ns;  // every mbarrier wait gives up after this long
+    int prefetch_w;          // 1: the W tiles of the first ring fill are requested before the dependency wait
 };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
@@ -117,14 +119,15 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 return false;
             }
@@ -377,9 +380,10 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             };
             // W is a constant of the model: fill the ring with its tiles before waiting for the kernel
-            // that produces the activations, then add the A tiles of those stages.
+            // that produces the activations, then add the A tiles of those stages.  (Not when W itself was
+            // written by work that may still be running: the host then clears prefetch_w for this launch.)
             int n_pref = 0;
-            for (KbCursor pre(p, MAX_BOXES); n_pref < STAGES && pre.valid; pre.advance(p, MAX_BOXES), ++n_pref) {
+            for (KbCursor pre(p, MAX_BOXES); p.prefetch_w && n_pref < STAGES && pre.valid; pre.advance(p, MAX_BOXES), ++n_pref) {
                 const uint32_t full = bar_full + 8 * n_pref;
                 const uint32_t sa = tiles + n_pref * STAGE_BYTES;
                 if (lane == 0) mbar_expect_tx(full, a_box_bytes + (uint32_t)(pre.nb * BOX_N * 128));
@@ -391,7 +395,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const uint32_t full = bar_full + 8 * stage;
                 const uint32_t sa = tiles + stage * STAGE_BYTES;
                 if (issued >= n_pref) {
-                    const bool got = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
+                    const bool got = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.wait_limit_ns);
                     if (!__all_sync(0xffffffffu, got)) {
                         ok = false;
                         break;
@@ -438,7 +442,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // dual: the tile takes both accumulator stages (one per m-tile), so tiles do not overlap
                     const bool dual = IS_ARGMAX && p.dual;
                     const uint32_t as = dual ? 0u : (tile & 1u), aphase = dual ? (tile & 1u) : ((tile >> 1) & 1u);
-                    if (!mbar_wait(bar_tempty + 8 * as, aphase ^ 1u, abort_flag)) {
+                    if (!mbar_wait(bar_tempty + 8 * as, aphase ^ 1u, abort_flag, p.wait_limit_ns)) {
                         ok = false;
                         break;
                     }
@@ -446,7 +450,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint32_t idesc = Q8 ? make_idesc_e4m3(nb * BOX_N) : make_idesc_bf16(nb * BOX_N);
                     const uint32_t d_tmem = tmem_base + as * ACC_COLS;
                     for (int kb = 0; kb < p.num_kb; ++kb) {
-                        if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) {
+                        if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.wait_limit_ns)) {
                             ok = false;
                             break;
                         }
@@ -520,7 +524,7 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < 8; ++c) sc[c] = (c * 32 + lane < n_valid) ? p.col_scale[col0 + c * 32 + lane] : 0.0f;
                 }
-                if (!mbar_wait(bar_tfull + 8 * as, aphase, abort_flag)) {
+                if (!mbar_wait(bar_tfull + 8 * as, aphase, abort_flag, p.wait_limit_ns)) {
                     ok = false;
                     break;
                 }
@@ -643,20 +647,41 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         if (IS_ARGMAX) {
             // The CTA that finishes last turns the merged keys into the outputs and re-arms the scratch.
+            // A CTA that gave up on a wait says so in the word after the ticket before it takes its
+            // ticket, so the last CTA knows that the merged keys are incomplete.
             const int et = threadIdx.x - 64;
             __threadfence();
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (et == 0) {
+                if (*abort_flag) {
+                    atomicAdd(p.ticket + 1, 1u);
+                    atomicOr(p.status, SPEC_STATUS_TIMEOUT);
+                    __threadfence();
+                }
                 const unsigned int t = atomicAdd(p.ticket, 1u);
-                *is_last = (t == gridDim.x - 1) ? 1 : 0;
+                int last = (t == gridDim.x - 1) ? 1 : 0;
+                if (last) {  // every other CTA has published by now: 2 = some CTA gave up
+                    __threadfence();
+                    if (*((volatile unsigned int*)(p.ticket + 1)) != 0u) last = 2;
+                }
+                *is_last = last;
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (*is_last) {
                 __threadfence();
+                const bool incomplete = *is_last == 2;
                 for (int i = et; i < p.a_rows; i += 128) {
                     const unsigned long long key = atomicExch(p.keys + i, 0ull);
                     int idx = (int)(~(uint32_t)(key & 0xFFFFFFFFull));
                     if (idx < 0 || idx >= p.V) idx = 0;
+                    if (incomplete) {  // some slice of the vocabulary is missing: no row may pass for a result
+                        if (p.keys_out) p.keys_out[i] = (long long)0x8000000000000000ull;  // below every real key
+                        else {
+                            p.argmax[i] = -1;
+                            if (p.maxv) p.maxv[i] = -INFINITY;
+                        }
+                        continue;
+                    }
                     if (p.keys_out) {
                         // shard of the vocabulary: global token id, and the sign bit flipped so that the key
                         // orders correctly as a signed 64-bit integer (what a max all-reduce compares)
@@ -667,8 +692,11 @@ head_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     p.argmax[i] = idx;
                     if (p.maxv) p.maxv[i] = from_orderable_f32((uint32_t)(key >> 32)) * (Q8 ? p.row_scale[i] : 1.0f);
                 }
-                if (et == 0) *p.ticket = 0u;
-                if (p.fuse_accept) {
+                if (et == 0) {
+                    p.ticket[0] = 0u;
+                    p.ticket[1] = 0u;
+                }
+                if (p.fuse_accept && !incomplete) {
                     // the predictions are complete: greedy acceptance right here saves a kernel launch
                     __threadfence();
                     asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -805,7 +833,8 @@ static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks, bool al
 }
 
 static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks, bool allow_dual = false) {
-    // Tuning aid: NGRAM_SPEC_SHAPE="box,group,chunks" overrides the choice (values are clamped).
+#ifdef NGRAM_SPEC_TUNING
+    // Tuning builds only: NGRAM_SPEC_SHAPE="box,group,chunks" overrides the choice (values are clamped).
     if (const char* ov = getenv("NGRAM_SPEC_SHAPE")) {
         int box = 32, g = 1, c = 1;
         if (sscanf(ov, "%d,%d,%d", &box, &g, &c) == 3 && (box == 16 || box == 32 || box == 64 || box == 128 || box == 256)) {
@@ -820,15 +849,20 @@ static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks, bool all
             return s;
         }
     }
-    static std::map<std::tuple<int, int, int, int, size_t, bool>, Shape> cache;
+#endif
+    // Process-wide table of the shapes chosen so far.
     const auto key = std::make_tuple(a_rows, ctx->V, ctx->d, ctx->num_sms, max_chunks, allow_dual);
+    std::lock_guard<std::mutex> lock(host_mutex());
+    static std::map<std::tuple<int, int, int, int, size_t, bool>, Shape> cache;
     auto it = cache.find(key);
     if (it != cache.end()) return it->second;
     Shape s = choose_shape(a_rows, ctx->V, ctx->num_sms, max_chunks, allow_dual);
     cache[key] = s;
+#ifdef NGRAM_SPEC_TUNING
     if (getenv("NGRAM_SPEC_TRACE"))
         fprintf(stderr, "[ngram_spec] rows=%d V=%d d=%d: dual=%d box=%d group=%d slots=%d chunks=%d grid=%d a_box=%d stages=%d stage=%dB smem=%dB\n",
                 a_rows, ctx->V, ctx->d, s.dual, s.box_n, s.group, s.n_slots, s.n_chunks, s.grid, s.a_box_rows, s.stages, s.stage_bytes, s.smem);
+#endif
     return s;
 }
 
@@ -848,6 +882,7 @@ static int w_map(spec_ctx* ctx, const WMaps** out, bool embedding = false) {
 template <int MODE, int KT>
 static int set_smem_attr(spec_ctx* ctx) {
     static bool done[64] = {false};
+    std::lock_guard<std::mutex> lock(host_mutex());
     bool& d = done[ctx->device & 63];
     if (d) return SPEC_OK;
     int rc = check_cuda(ctx, cudaFuncSetAttribute(head_gemm_kernel<MODE, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT),
@@ -890,6 +925,8 @@ static void fill_common(spec_ctx* ctx, GemmParams& p, int a_rows, const Shape& s
     p.idx_offset = 0;
     p.col_scale = nullptr;
     p.row_scale = nullptr;
+    p.wait_limit_ns = WAIT_LIMIT_NS;
+    p.prefetch_w = 1;
 }
 
 int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, cudaStream_t st,
@@ -998,6 +1035,10 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
     p.maxv = d_max;
     p.col_scale = ctx->wscale;
     p.row_scale = d_hscale;
+    // The 8-bit head may have been written by a kernel of this stream that is still running (it lets its
+    // dependents start early): the first verification after a head was set reads W only after the wait.
+    p.prefetch_w = ctx->wq_fresh ? 0 : 1;
+    ctx->wq_fresh = false;
     cudaError_t e = launch_pdl(head_gemm_kernel<MODE_ARGMAX_Q8, 1>, dim3(sh.grid), dim3(GEMM_THREADS), (size_t)sh.smem, st, *tmA, *tmA2,
                                ctx->tm_q, p);
     ctx->launches += 1;
@@ -1020,20 +1061,19 @@ int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cud
     return check_cuda(ctx, cudaGetLastError(), "spec_debug_logits launch");
 }
 
-int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_t* d_tab_idx, float* d_tab_val,
-                 int32_t* d_ext, cudaStream_t st) {
+// Table rows for the n_rows rows of A that start at d_rows (the whole matrix, or one rank's slice of it).
+int launch_table(spec_ctx* ctx, const void* d_rows, int n_rows, int k_tab, int32_t* d_tab_idx, float* d_tab_val, cudaStream_t st) {
     const int kt = k_tab <= 8 ? 8 : (k_tab <= 16 ? 16 : 32);
     int rc = kt == 8 ? set_smem_attr<MODE_TOPK, 8>(ctx) : (kt == 16 ? set_smem_attr<MODE_TOPK, 16>(ctx) : set_smem_attr<MODE_TOPK, 32>(ctx));
     if (rc) return rc;
-    const int V = ctx->V;
     // partial lists cost 8 bytes per entry and chunk: keep them under 256 MB
-    int max_chunks = (int)std::max<long long>(1, (256ll << 20) / ((long long)V * k_tab * 8));
-    const Shape sh = cached_shape(ctx, V, (size_t)max_chunks);
+    int max_chunks = (int)std::max<long long>(1, (256ll << 20) / ((long long)n_rows * k_tab * 8));
+    const Shape sh = cached_shape(ctx, n_rows, (size_t)max_chunks);
     const WMaps* tmW;
     if ((rc = w_map(ctx, &tmW))) return rc;
     CUtensorMap tmA;
-    if ((rc = make_tensor_map(ctx, &tmA, d_rows, V, ctx->d, sh.a_box_rows))) return rc;
-    const size_t need = (size_t)sh.n_chunks * V * k_tab;
+    if ((rc = make_tensor_map(ctx, &tmA, d_rows, n_rows, ctx->d, sh.a_box_rows))) return rc;
+    const size_t need = (size_t)sh.n_chunks * n_rows * k_tab;
     if (need > ctx->part_capacity) {
         cudaStreamSynchronize(st);
         cudaFree(ctx->d_part_val);
@@ -1046,7 +1086,7 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
         ctx->part_capacity = need;
     }
     GemmParams p;
-    fill_common(ctx, p, V, sh);
+    fill_common(ctx, p, n_rows, sh);
     p.k_tab = k_tab;
     p.part_val = ctx->d_part_val;
     p.part_idx = ctx->d_part_idx;
@@ -1057,17 +1097,44 @@ int launch_table(spec_ctx* ctx, const void* d_rows, int k_tab, int w_ext, int32_
     else
         head_gemm_kernel<MODE_TOPK, 32><<<sh.grid, GEMM_THREADS, sh.smem, st>>>(tmA, tmA, *tmW, p);
     if ((rc = check_cuda(ctx, cudaGetLastError(), "build_model_ngram_tables launch"))) return rc;
-    merge_topk_kernel<<<(V + 127) / 128, 128, 0, st>>>(ctx->d_part_val, ctx->d_part_idx, sh.n_chunks, V, k_tab, d_tab_idx,
-                                                      d_tab_val);
+    merge_topk_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(ctx->d_part_val, ctx->d_part_idx, sh.n_chunks, n_rows, k_tab, d_tab_idx,
+                                                           d_tab_val);
     ctx->launches += 2;
-    if ((rc = check_cuda(ctx, cudaGetLastError(), "table merge launch"))) return rc;
-    if (d_ext) {
-        const long long n = (long long)V * k_tab;
-        extend_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d_tab_idx, V, k_tab, w_ext, d_ext);
-        ctx->launches += 1;
-        if ((rc = check_cuda(ctx, cudaGetLastError(), "table extension launch"))) return rc;
+    return check_cuda(ctx, cudaGetLastError(), "table merge launch");
+}
+
+int launch_extend_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, int w_ext, int32_t* d_ext, cudaStream_t st) {
+    const long long n = (long long)ctx->V * k_tab;
+    extend_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d_tab_idx, ctx->V, k_tab, w_ext, d_ext);
+    ctx->launches += 1;
+    return check_cuda(ctx, cudaGetLastError(), "table extension launch");
+}
+
+// ------------------------------------------------------------------------------------------ bounded-wait check
+// Test aid: one thread waits, with the same bounded wait the contraction uses, on an mbarrier that nobody
+// ever arrives at.  The wait must give up after limit_ns, the kernel must return, and the context must
+// report SPEC_STATUS_TIMEOUT.  With mark_incomplete the kernel also does what a contraction CTA does when
+// it gives up: it counts itself in the word after the merge ticket, so that the next verification finds
+// its merge incomplete.
+__global__ void wait_probe_kernel(unsigned long long limit_ns, int* status, unsigned int* ticket, int mark_incomplete) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool got = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_ns);
+        if (!got) {
+            atomicOr(status, SPEC_STATUS_TIMEOUT);
+            if (mark_incomplete) atomicAdd(ticket + 1, 1u);
+        }
     }
-    return SPEC_OK;
+}
+
+int launch_wait_probe(spec_ctx* ctx, unsigned long long limit_ns, int mark_incomplete, cudaStream_t st) {
+    wait_probe_kernel<<<1, 32, 0, st>>>(limit_ns, ctx->d_status, ctx->d_ticket, mark_incomplete);
+    ctx->launches += 1;
+    return check_cuda(ctx, cudaGetLastError(), "spec_debug_expire_wait launch");
 }
 
 // ------------------------------------------------------------------------------------------ vocabulary shards
@@ -1211,17 +1278,25 @@ int launch_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2,
 }  // namespace ngs
 
 // ------------------------------------------------------------------------------------------ allocation-free verify
-// Scratch of verify_lmhead_argmax_noalloc: merge keys for SPEC_NOALLOC_MAX_ROWS rows, then one word
-// for the completion ticket and one for the status bits.  It lives in the library image, so every
-// GPU that loads the library holds these ~33 KB until the process exits.
+// Scratch of verify_lmhead_argmax_noalloc: merge keys for SPEC_NOALLOC_MAX_ROWS rows, then one 64-bit
+// word holding the completion ticket and the count of CTAs that gave up, and one for the status bits.
+// It lives in the library image, so every GPU that loads the library holds these ~33 KB until the
+// process exits.
 static __device__ __align__(256) unsigned long long g_noalloc_scratch[SPEC_NOALLOC_MAX_ROWS + 32];
 
 namespace ngs {
 struct NoAllocDevice {
+    std::mutex lock;  // host-side state below; calls on one device are enqueued one at a time
     bool ready = false;
     unsigned long long* scratch = nullptr;  // device address of g_noalloc_scratch on this device
     int num_sms = 0;
     EncodeTiledFn encode = nullptr;
+    // tensor maps of the head seen last, so that a decode loop does not re-encode them on every call
+    const void* w_base = nullptr;
+    int w_V = 0, w_d = 0;
+    WMaps tm_w;
+    spec_ctx::AMap a_maps[4];
+    int a_map_next = 0;
 };
 static NoAllocDevice g_noalloc_dev[64];
 }  // namespace ngs
@@ -1242,6 +1317,7 @@ extern "C" int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d,
     if (e != cudaSuccess) return check_cuda(nullptr, e, "verify_lmhead_argmax_noalloc: cudaSetDevice");
 
     NoAllocDevice& nd = g_noalloc_dev[device];
+    std::lock_guard<std::mutex> guard(nd.lock);
     if (!nd.ready) {
         // One-time set-up for this device (made current above).  In host code the array's name is only a
         // handle: the address a kernel can use has to be asked for, per device.
@@ -1275,6 +1351,12 @@ extern "C" int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d,
     tmp.d_keys = nd.scratch;
     tmp.d_ticket = reinterpret_cast<unsigned int*>(nd.scratch + SPEC_NOALLOC_MAX_ROWS);
     tmp.d_status = reinterpret_cast<int*>(nd.scratch + SPEC_NOALLOC_MAX_ROWS + 1);
+    if (nd.w_base == d_unembed && nd.w_V == V && nd.w_d == d) {  // same head as last time: reuse its tensor maps
+        tmp.tm_w = nd.tm_w;
+        tmp.tm_w_ready = true;
+        for (int i = 0; i < 4; ++i) tmp.a_maps[i] = nd.a_maps[i];
+        tmp.a_map_next = nd.a_map_next;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     int rc = SPEC_OK;
     {
@@ -1287,5 +1369,11 @@ extern "C" int verify_lmhead_argmax_noalloc(const void* d_unembed, int V, int d,
     }
     if (rc == SPEC_OK) rc = launch_verify(&tmp, d_hidden, M, d_argmax, d_max, st, nullptr, nullptr, 0);
     if (rc != SPEC_OK) return fail(nullptr, rc, "%s", tmp.err);
+    nd.w_base = d_unembed;
+    nd.w_V = V;
+    nd.w_d = d;
+    nd.tm_w = tmp.tm_w;
+    for (int i = 0; i < 4; ++i) nd.a_maps[i] = tmp.a_maps[i];
+    nd.a_map_next = tmp.a_map_next;
     return SPEC_OK;
 }

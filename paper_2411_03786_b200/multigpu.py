@@ -55,6 +55,38 @@ def sharded_verify(ctx, hidden, vocab_offset: int, V_total: int, with_max: bool 
     return unpack_keys(keys, V_total, with_max)
 
 
+def all_gather_rows(local: torch.Tensor, n_total: int, rank: int, world: int) -> torch.Tensor:
+    """Stitches per-rank row slices (rank r owns ``shard_sequences(n_total, r, world)``) into the whole
+    ``[n_total, ...]`` array on every rank: one all-gather of equally padded slices, into local buffers."""
+    import torch.distributed as dist
+    first, count = shard_sequences(n_total, rank, world)
+    assert local.shape[0] == count, "this rank's slice has the wrong number of rows"
+    if not (dist.is_available() and dist.is_initialized()) or world == 1:
+        return local.clone()
+    most = (n_total + world - 1) // world
+    padded = torch.zeros((most,) + tuple(local.shape[1:]), dtype=local.dtype, device=local.device)
+    padded[:count] = local
+    parts = [torch.empty_like(padded) for _ in range(world)]
+    dist.all_gather(parts, padded)
+    return torch.cat([parts[r][:shard_sequences(n_total, r, world)[1]] for r in range(world)], dim=0)
+
+
+def sharded_table_build(ctx, k_tab: int, w_ext: int, rank: int, world: int, rows: torch.Tensor | None = None):
+    """Model bigram table with the rows split over the ranks (every rank holds the whole head):
+    each rank contracts its ``V / world`` rows, one all-gather of the ``[rows, k_tab]`` int32 slices
+    gives every rank the complete table, and the extension is then derived locally.
+    Returns ``(table[V, k_tab], ext[V, k_tab, w_ext] or None)``; the context adopts them when w_ext > 0."""
+    V = ctx.V
+    first, count = shard_sequences(V, rank, world)
+    tab = torch.zeros((V, k_tab), dtype=torch.int32, device=ctx._keep[0].device)
+    ctx.build_model_ngram_table_rows(k_tab, first, count, tab, rows=rows)
+    whole = all_gather_rows(tab[first:first + count].contiguous(), V, rank, world)
+    if w_ext > 0:
+        return whole, ctx.extend_model_table(whole, w_ext)
+    ctx.set_model_table(whole)
+    return whole, None
+
+
 def pack_key(value: float, token_id: int) -> int:
     """Host-side statement of the shard key format (for tests and debugging): a signed 64-bit integer
     that is larger for a larger fp32 logit and, for equal logits, for a smaller token id."""

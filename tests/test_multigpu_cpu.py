@@ -105,3 +105,42 @@ def test_max_all_reduce_of_shard_keys_picks_the_global_argmax():
         v, i = multigpu.unpack_key(k0[j])
         want = (v0[j], i0[j]) if (v0[j] > v1[j] or (v0[j] == v1[j] and i0[j] < i1[j])) else (v1[j], i1[j])
         assert (v, i) == (np.float32(want[0]), want[1])
+
+
+def _table_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    import synth
+    V, d, k = 37, 16, 3                                   # odd V: the two slices differ in size
+    E = synth.gaussian_weights(V, d, 1.0, 3, "E")
+    W = synth.gaussian_weights(V, d, 1.0, 3, "W")
+    first, count = multigpu.shard_sequences(V, rank, world)
+    mine, _ = oracle.model_table(E, W, k, rows=np.arange(first, first + count))     # this rank's rows only
+    whole = multigpu.all_gather_rows(torch.from_numpy(mine), V, rank, world)
+    out.put((rank, whole.numpy().tolist()))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_stitch_their_table_slices_into_the_whole_table():
+    import oracle
+    import synth
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_table_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    E = synth.gaussian_weights(37, 16, 1.0, 3, "E")
+    W = synth.gaussian_weights(37, 16, 1.0, 3, "W")
+    whole, _ = oracle.model_table(E, W, 3)
+    assert res[0][1] == res[1][1] == whole.tolist()
+    # single process: the slice is the table
+    one = multigpu.all_gather_rows(torch.from_numpy(whole), 37, 0, 1)
+    assert one.numpy().tolist() == whole.tolist()

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import synth
 from gpu_util import dev_bf16
 
@@ -26,7 +27,8 @@ def test_noalloc_verify_matches_context_verify_on_two_calls_in_a_row():
     dW = dev_bf16(W)
     ctx = ngs.SpecContext(dW, dW)
     for call, M in enumerate((300, 77, 200)):   # later calls reuse the scratch the earlier ones left behind; all three row regimes
-        dH = dev_bf16(synth.hidden_literal(M, d, seed=50 + call))
+        H = synth.hidden_literal(M, d, seed=50 + call)
+        dH = dev_bf16(H)
         ref_am, ref_mx = ctx.verify_lmhead_argmax(dH, with_max=True)
         out = (torch.empty(M, dtype=torch.int32, device="cuda"), torch.empty(M, dtype=torch.float32, device="cuda"))
         allocs = lambda: torch.cuda.memory_stats()["allocation.all.allocated"]   # cumulative, frees do not lower it
@@ -37,6 +39,12 @@ def test_noalloc_verify_matches_context_verify_on_two_calls_in_a_row():
         assert torch.equal(am, ref_am)                       # same kernel, integer result: identical
         assert (mx - ref_mx).abs().max().item() <= TOL
         assert (am >= 0).all() and (am < V).all()
+        # and against the CPU oracle, on a seeded sample of rows (first, last, tile edges)
+        rows = np.array(sorted({0, 1, M - 1, min(127, M - 1), min(128, M - 1)} | set(np.random.default_rng(call).integers(0, M, 24).tolist())))
+        o_am, o_mx, gap = oracle.verify(H, W, rows=rows)
+        bad = am.cpu().numpy()[rows] != o_am
+        assert not (bad & (gap >= TOL)).any()
+        assert np.abs(mx.cpu().numpy()[rows].astype(np.float64) - o_mx).max() <= TOL
     ctx.close()
 
 
