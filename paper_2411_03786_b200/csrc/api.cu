@@ -148,6 +148,8 @@ int spec_init(spec_ctx** out, const void* d_embed, const void* d_unembed, int dt
         if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_keys, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS),
                              "cudaMalloc(keys)"))) break;
         if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_ticket, 2 * sizeof(unsigned int)), "cudaMalloc(ticket)"))) break;
+        if ((rc = check_cuda(nullptr, cudaMalloc(&ctx->d_draft_work, 2 * sizeof(unsigned int)), "cudaMalloc(draft work counter)"))) break;
+        cudaMemsetAsync(ctx->d_draft_work, 0, 2 * sizeof(unsigned int), st);
         cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st);
         cudaMemsetAsync(ctx->d_keys, 0, sizeof(unsigned long long) * SPEC_MAX_VERIFY_ROWS, st);
         cudaMemsetAsync(ctx->d_ticket, 0, 2 * sizeof(unsigned int), st);
@@ -174,6 +176,7 @@ int spec_destroy(spec_ctx* ctx) {
     cudaFree(ctx->d_status);
     cudaFree(ctx->d_keys);
     cudaFree(ctx->d_ticket);
+    cudaFree(ctx->d_draft_work);
     cudaFree(ctx->d_centred);
     cudaFree(ctx->d_colsum);
     cudaFree(ctx->d_part_val);

@@ -42,6 +42,7 @@ struct spec_ctx {
     // verify merge scratch: one packed (value, ~index) key per row + completion ticket
     unsigned long long* d_keys = nullptr;
     unsigned int* d_ticket = nullptr;  // [0] CTAs finished, [1] CTAs that gave up on a bounded wait
+    unsigned int* d_draft_work = nullptr;  // batch drafting: [0] next sequence to take, [1] CTAs that have left
     // table-build scratch: partial top-k lists per vocabulary chunk
     float* d_part_val = nullptr;
     int32_t* d_part_idx = nullptr;

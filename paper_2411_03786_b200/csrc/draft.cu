@@ -1,6 +1,7 @@
-// Context N-gram drafting and mixed allocation: one CTA per sequence, or for long histories one
-// thread-block cluster per sequence whose CTAs each scan a slice of the history and group their
-// matches in the leader CTA's hash table through distributed shared memory.
+// Context N-gram drafting and mixed allocation, latency path: one CTA per sequence, or for long
+// histories one thread-block cluster per sequence whose CTAs each scan a slice of the history and group
+// their matches in the leader CTA's hash table through distributed shared memory.  (Batches of many
+// sequences take the team kernel in draft_team.cu.)
 //
 // One streaming pass over the history serves every query length at once.  A position p is the
 // start of a continuation for query length q when the q tokens before p equal the last q tokens
@@ -14,66 +15,15 @@
 // A history of up to 8192 tokens is first copied into shared memory (one round of 128-bit loads);
 // the scan, the key comparisons and the candidate rows then never wait for global memory again,
 // which is what the latency of a single short sequence is made of.
-//
-// On the throughput path (one CTA per sequence, history read from global memory) the scan itself only
-// looks for matches: per 128-bit vector one comparison chain, per warp iteration
-// (512 tokens) one vote.  Where a match turns up its position goes into a per-warp queue, and a
-// queue-full of matches is grouped at once, one per lane, so that the dependent reads each match
-// needs (suffix, continuation, the group's representative) overlap instead of stalling the scan.
 #include <cooperative_groups.h>
 
-#include "common.cuh"
+#include "draft_common.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace ngs {
 
-struct DraftParams {
-    const int32_t* hist;
-    const int32_t* len;
-    int S, cap;
-    int qs[kMaxNQ];
-    int n_q, q_max, q_min;
-    int topk, B, w, flags;
-    const int32_t* tab;
-    int k_tab;
-    const int32_t* ext;
-    int w_ext;
-    int V;
-    int32_t* drafts;
-    int32_t* ndrafts;
-    int32_t* src;
-    int32_t* counts;
-    int* status;
-    int slots;       // hash table size (power of two)
-    int max_groups;  // slots / 2
-    int stage_hist;  // 1: copy the history into shared memory first (single CTA, short history)
-    int hist_off;    // where that copy lives, in ints from the start of the hash table
-    int queue_off;   // byte offset of the per-warp match queues from the start of dynamic shared memory
-};
-
-constexpr int kMaxPasses = 1024;
 constexpr int kRankMax = 512;                          // groups ranked by counting (all threads) up to here
-constexpr int kMaxCand = kMaxNQ * kMaxB + kMaxKTab;    // candidate rows before duplicates are dropped
-constexpr int kMatchQueue = 128;                       // matches a warp queues before it groups them
-
-__device__ __forceinline__ uint32_t fmix32(uint32_t h) {
-    h ^= h >> 16;
-    h *= 0x85EBCA6Bu;
-    h ^= h >> 13;
-    h *= 0xC2B2AE35u;
-    h ^= h >> 16;
-    return h;
-}
-
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        unsigned long long other = __shfl_xor_sync(0xffffffffu, v, o);
-        v = other > v ? other : v;
-    }
-    return v;
-}
 
 struct DraftSmem {
     unsigned long long run_key[kMaxNQ][kMaxB];  // per query length: ranked (count << 32 | start) keys
@@ -95,55 +45,8 @@ struct DraftSmem {
     int n_out;
 };
 
-// Group the match whose continuation starts at p (query index qi).
-__device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int p, int qi, int key_len, uint32_t hsh,
-                                             int slots, int max_groups, int* rep, int* cnt, int* last,
-                                             int* grp_slot, DraftSmem* sm) {
-    if (*((volatile int*)&sm->overflow)) return;  // this pass is void already: do not fill the table further
-    uint32_t slot = hsh & (uint32_t)(slots - 1);
-    const int me = (qi << 28) | p;
-    for (int probe = 0; probe < slots; ++probe) {
-        int cur = *((volatile int*)&rep[slot]);
-        if (cur == -1) {
-            int old = atomicCAS(&rep[slot], -1, me);
-            if (old == -1) {
-                int g = atomicAdd(&sm->n_groups, 1);
-                if (g >= max_groups) {
-                    sm->overflow = 1;
-                    return;
-                }
-                grp_slot[g] = (int)slot;
-                atomicAdd(&cnt[slot], 1);
-                atomicMax(&last[slot], p);
-                return;
-            }
-            cur = old;
-        }
-        if ((cur >> 28) == qi) {
-            const int rp = cur & 0x0FFFFFFF;
-            bool same = true;
-            for (int t = 0; t < key_len; ++t)
-                if (h[rp + t] != h[p + t]) {
-                    same = false;
-                    break;
-                }
-            if (same) {
-                atomicAdd(&cnt[slot], 1);
-                atomicMax(&last[slot], p);
-                return;
-            }
-        }
-        slot = (slot + 1) & (uint32_t)(slots - 1);
-    }
-    sm->overflow = 1;
-}
-
-// STREAM = false: the latency path - a short history staged in shared memory (one CTA; a decode step's
-// drafting latency, so this instantiation carries nothing it does not execute), or a long history split
-// over a cluster (few sequences: matches are grouped where they are found, which also notices a full
-// table at once and cuts a void pass short).
-// STREAM = true: the throughput path - one CTA per sequence reading its history from global memory.
-template <bool STREAM>
+// The kernel carries nothing it does not execute: a decode step's drafting latency is sensitive to its
+// code size (a quarter of it is cold instruction fetch).
 __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DraftSmem* sm = reinterpret_cast<DraftSmem*>(smem_raw);
@@ -158,13 +61,11 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     cg::cluster_group cluster = cg::this_cluster();
     const int csize = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
     const bool leader = crank == 0;
-    // (the throughput path addresses its table directly: a mapped address takes the cluster's path even to itself)
-    const bool direct = STREAM;
-    DraftSmem* lsm = direct ? sm : cluster.map_shared_rank(sm, 0);
-    int* lrep = direct ? rep : cluster.map_shared_rank(rep, 0);
-    int* lcnt = direct ? cnt : cluster.map_shared_rank(cnt, 0);
-    int* llast = direct ? last : cluster.map_shared_rank(last, 0);
-    int* lgrp_slot = direct ? grp_slot : cluster.map_shared_rank(grp_slot, 0);
+    DraftSmem* lsm = cluster.map_shared_rank(sm, 0);
+    int* lrep = cluster.map_shared_rank(rep, 0);
+    int* lcnt = cluster.map_shared_rank(cnt, 0);
+    int* llast = cluster.map_shared_rank(last, 0);
+    int* lgrp_slot = cluster.map_shared_rank(grp_slot, 0);
 
     // barrier over all CTAs of the sequence (a plain CTA barrier when there is only one: much cheaper)
     auto pass_sync = [&]() {
@@ -258,7 +159,6 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     const int n_vec_all = (max(n_scan, 0) + 3) >> 2;
     const int v_chunk = (n_vec_all + csize - 1) / csize;  // this CTA's slice of the history
     const int n_vec = min(n_vec_all, (crank + 1) * v_chunk);
-    int* wq = reinterpret_cast<int*>(smem_raw + P.queue_off) + warp * kMatchQueue;  // this warp's queue of matches
 
     int R = 1;
     bool gave_up = false;
@@ -313,55 +213,15 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                     if (m < q || L < q + w) continue;
                     const uint32_t hq = fmix32(hc + (uint32_t)qi * 0x632BE5ABu);
                     if (R > 1 && (int)(fmix32(hq ^ 0xA511E9B3u) % (uint32_t)R) != r) continue;
-                    insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, lrep, lcnt, llast, lgrp_slot, lsm);
+                    insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, lrep, lcnt, llast, lgrp_slot, &lsm->n_groups, &lsm->overflow);
                 }
             };
-            // Matches are not grouped where they are found: a match costs a chain of dependent reads of
-            // the history (suffix, continuation, the group's representative), and a warp that stopped
-            // for each one would scan at the speed of that chain.  The warp queues the positions and
-            // groups a queue-full at a time, one match per lane, so the chains of 32 matches overlap.
-            int qn = 0;  // queued matches (the same in every lane)
-            auto flush_matches = [&]() {
-                __syncwarp();
-                for (int i = lane; i < qn; i += 32) handle_match(wq[i]);
-                __syncwarp();
-                qn = 0;
-            };
-            // v0 = the lane's first vector, its u-th vector is v0 + u * ustride
+            // v0 = the lane's first vector, its u-th vector is v0 + u * ustride; a match is grouped where it is found
             auto handle_hits = [&](unsigned hits, int v0, int ustride) {
-                if constexpr (!STREAM) {
-                    while (hits) {
-                        const int bit = __ffs(hits) - 1;
-                        hits &= hits - 1;
-                        handle_match(((v0 + (bit >> 2) * ustride) << 2) + (bit & 3));
-                    }
-                    return;
-                } else {
-                if (!__any_sync(0xffffffffu, hits != 0u)) return;
-                const int nh = __popc(hits);
-                int incl = nh;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                const int total = __shfl_sync(0xffffffffu, incl, 31);
-                if (total > kMatchQueue) {  // denser than the queue: group them in place
-                    while (hits) {
-                        const int bit = __ffs(hits) - 1;
-                        hits &= hits - 1;
-                        handle_match(((v0 + (bit >> 2) * ustride) << 2) + (bit & 3));
-                    }
-                    return;
-                }
-                if (qn + total > kMatchQueue) flush_matches();
-                int at = qn + incl - nh;
                 while (hits) {
                     const int bit = __ffs(hits) - 1;
                     hits &= hits - 1;
-                    wq[at++] = ((v0 + (bit >> 2) * ustride) << 2) + (bit & 3);
-                }
-                qn += total;
+                    handle_match(((v0 + (bit >> 2) * ustride) << 2) + (bit & 3));
                 }
             };
             // 128-bit loads, four per thread in flight.  The common case (no match among the warp's
@@ -372,39 +232,25 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
                 if (__any_sync(0xffffffffu, *((volatile int*)&lsm->overflow))) break;
                 const int v0 = vw + lane;
                 int4 vv[4];
-                int left[4];  // token before the vector: lane 0 asks for it together with the vectors
+                int left[4];  // token before the vector
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int vi = v0 + u * nthr;
                     vv[u] = (vi < n_vec) ? h4[vi] : make_int4(-3, -3, -3, -3);
-                    if constexpr (STREAM) left[u] = (need2 && lane == 0 && vi > 0 && vi < n_vec) ? h[(vi << 2) - 1] : -5;
                 }
-                if constexpr (!STREAM) {
-                    if (need2) {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int vi = v0 + u * nthr;
-                            left[u] = __shfl_up_sync(0xffffffffu, vv[u].w, 1);
-                            if (lane == 0) left[u] = (vi > 0 && vi < n_vec) ? h[(vi << 2) - 1] : -5;
-                        }
-                    }
-                } else if (need2) {  // token before each position: from this vector, or from the lane to the left
-                    bool some = false;
+                if (need2) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const int up = __shfl_up_sync(0xffffffffu, vv[u].w, 1);
-                        if (lane != 0) left[u] = up;
-                        some = some || (vv[u].x == t0 && left[u] == t1) || (vv[u].y == t0 && vv[u].x == t1) ||
-                               (vv[u].z == t0 && vv[u].y == t1) || (vv[u].w == t0 && vv[u].z == t1);
+                        const int vi = v0 + u * nthr;
+                        left[u] = __shfl_up_sync(0xffffffffu, vv[u].w, 1);
+                        if (lane == 0) left[u] = (vi > 0 && vi < n_vec) ? h[(vi << 2) - 1] : -5;
                     }
-                    if (!__any_sync(0xffffffffu, some)) continue;
                 }
                 unsigned hits = 0;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) hits |= vec_hits(vv[u], left[u], (v0 + u * nthr) << 2) << (4 * u);
                 handle_hits(hits, v0, nthr);
             }
-            if constexpr (STREAM) flush_matches();
             pass_sync();  // every CTA's matches are in the table
             const int ov = *((volatile int*)&lsm->overflow);
             pass_sync();  // every CTA has read the flag before the leader may reset it
@@ -662,14 +508,6 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     int slots = 1024;  // at most slots / 2 distinct continuations are grouped in one pass
     while (slots < cap / 2 && slots < 8192) slots <<= 1;
     int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);
-    // A batch that fills the GPU more than once runs faster with two or three CTAs per SM (the scan of one
-    // overlaps the barriers and serial phases of another): half the threads, and half the table where few
-    // groups are expected (every query has two tokens or more, or the history is short).  Measured on
-    // S x L = 592 x 32768, 592 x 131072 and 2048 x 8192: 1.9x, 1.1x and 2.3x faster than the shape above.
-    if (S > ctx->num_sms && cap > 8192 && (P.q_min >= 2 || cap <= 16384)) {
-        threads = 512;
-        if (slots > 4096) slots = 4096;
-    }
 #ifdef NGRAM_SPEC_TUNING
     // Tuning builds only: NGRAM_SPEC_DRAFT_SHAPE="threads,slots" overrides the choice (values are clamped).
     if (const char* ov = getenv("NGRAM_SPEC_DRAFT_SHAPE")) {
@@ -680,36 +518,41 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
         }
     }
 #endif
-    P.slots = slots;
-    P.max_groups = slots / 2;
     // CTAs per sequence: one per 16K tokens of capacity, at most 8, and only while the batch alone
-    // cannot fill the GPU (with many sequences one CTA each is the faster way to stream them)
+    // cannot fill the GPU (with many sequences the team kernel streams them)
     unsigned csize = 1;
     while (csize < 8 && (int)(csize * 2) * 16384 <= cap && (long long)S * (csize * 2) <= ctx->num_sms) csize <<= 1;
+    const bool stage = csize == 1 && cap <= 8192;
+    if (csize == 1) {
+        // Batches: histories of up to 16384 tokens are staged in shared memory by warp teams (when the batch
+        // fills the GPU more than twice over, or a history is too long for the staging of this kernel);
+        // longer ones are streamed by the scanner / finisher kernel.
+        const bool batch = S > 2 * ctx->num_sms;
+        if (cap <= 16384 && (batch || !stage)) {
+            const int rc = launch_draft_team(ctx, P, st);
+            if (rc != kDraftNoFit) return rc;  // (the largest draft shapes leave no room for the staged history)
+        }
+        if (!stage) return launch_draft_stream(ctx, P, st);
+    }
+    P.slots = slots;
+    P.max_groups = slots / 2;
     const size_t table_bytes = (size_t)slots * 3 * sizeof(int) + (size_t)P.max_groups * sizeof(int);
     const size_t cand_bytes = (size_t)(n_q * topk + kMaxKTab) * w * sizeof(int32_t);  // aliases the table
     const size_t work_bytes = ((table_bytes > cand_bytes ? table_bytes : cand_bytes) + 15) & ~size_t(15);
-    P.stage_hist = (csize == 1 && cap <= 8192) ? 1 : 0;
+    P.stage_hist = stage ? 1 : 0;
     P.hist_off = (int)(work_bytes / sizeof(int));
-    size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + work_bytes + (P.stage_hist ? (size_t)cap * sizeof(int32_t) : 0);
-    const bool throughput = !P.stage_hist && csize == 1;  // which instantiation runs (see draft_kernel)
-    P.queue_off = (int)((smem + 15) & ~size_t(15));
-    if (throughput) smem = (size_t)P.queue_off + (size_t)(threads / 32) * kMatchQueue * sizeof(int);  // per-warp match queues
+    const size_t smem = ((sizeof(DraftSmem) + 15) & ~size_t(15)) + work_bytes + (P.stage_hist ? (size_t)cap * sizeof(int32_t) : 0);
     static bool attr_set[64] = {false};
     std::unique_lock<std::mutex> lock(host_mutex());
     bool& attr_done = attr_set[ctx->device & 63];
     if (!attr_done) {
-        int rc = check_cuda(ctx, cudaFuncSetAttribute(draft_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024),
+        int rc = check_cuda(ctx, cudaFuncSetAttribute(draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024),
                             "draft: cudaFuncSetAttribute");
-        if (rc) return rc;
-        rc = check_cuda(ctx, cudaFuncSetAttribute(draft_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024),
-                        "draft: cudaFuncSetAttribute");
         if (rc) return rc;
         attr_done = true;
     }
     lock.unlock();
-    cudaError_t e = launch_pdl_cluster(throughput ? draft_kernel<true> : draft_kernel<false>, dim3((unsigned)S * csize),
-                                       dim3(threads), smem, st, csize, P);
+    cudaError_t e = launch_pdl_cluster(draft_kernel, dim3((unsigned)S * csize), dim3(threads), smem, st, csize, P);
     ctx->launches += 1;
     return check_cuda(ctx, e, "draft_context_ngrams launch");
 }

@@ -60,10 +60,10 @@ def test_random_draft_problem(ctx, case):
                                                  (V, [2], 9500, 1), (2, [4, 3], 8400, 5), (6, [1], 16000, 3),
                                                  (40, [1, 2], 10000, 2)])
 def test_batch_of_unstaged_histories(ctx, alpha, qs, Lmax, flags):
-    """More sequences than SMs, histories too long to stage in shared memory: the batch launch shape
-    (several CTAs per SM, smaller table) and the queued grouping of matches, from a few matches per
-    warp iteration (queue filled and flushed in mid-scan) to more than a queue holds (grouped in place);
-    the last case has more distinct continuations than the smaller table groups in one pass."""
+    """More sequences than SMs, histories of 8K to 17K tokens: the batch kernels (a team of 16 warps per CTA
+    up to 16384 tokens, scanner / finisher warps beyond) and the queued grouping of matches, from a few
+    matches per warp iteration (queue filled and flushed in mid-scan) to more than a queue holds (grouped
+    in place); some cases have more distinct continuations than the table groups in one pass."""
     g = np.random.default_rng(31000 + alpha + Lmax)
     S, B, w, topk, k_tab = 160, 12, 5, 6, 4
     cap = Lmax + 8
@@ -81,4 +81,46 @@ def test_batch_of_unstaged_histories(ctx, alpha, qs, Lmax, flags):
     got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, flags)
     for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
         assert np.array_equal(a.cpu().numpy(), b), name
+    assert ctx.get_status() == 0
+
+
+@pytest.mark.parametrize("S,Lmax,alpha,qs,flags", [
+    (2400, 2000, 6, [1], 3),         # one warp per sequence, per-warp tables; q = 1 on 6 symbols overflows them (several passes)
+    (2400, 300, 40, [3, 2, 1], 3),   # one warp per sequence, a handful of matches each
+    (1200, 900, 3, [2, 1], 7),       # two warps per sequence, grouping by the next token only
+    (1200, 5000, V, [2], 1),         # ... vocabulary-sized alphabet: hardly any match
+    (600, 1500, 6, [4, 3], 5),       # four warps per sequence
+    (600, 7000, 6, [1, 2], 3),       # ... about a thousand matches with several hundred distinct continuations: several passes
+    (320, 3000, 40, [2, 1], 2),      # eight warps per sequence, no duplicate removal
+    (310, 9000, 6, [3, 2], 3),       # eight warps by the batch, unstaged history
+    (300, 40000, 6, [2], 3),         # histories too long to stage: scanner and finisher warps, two tables
+    (200, 30000, 10, [1, 2], 3),     # ... with more distinct continuations than a table holds: several hand-overs per sequence
+    (150, 17000, 40, [3, 1], 7),     # ... fewer sequences than a CTA per SM could take twice
+])
+def test_batches_across_team_sizes(ctx, S, Lmax, alpha, qs, flags):
+    """Batches that fill the GPU more than twice over take the persistent kernels: warp teams (1, 2, 4, 8 or 16 warps,
+    by batch size) that stage a history of up to 16384 tokens in shared memory, scanner / finisher warps for longer
+    ones; sequences are pulled from a queue, and ragged lengths (down to empty) make the teams take different numbers
+    of them.  Two calls in a row: the work queue has to re-arm itself."""
+    import paper_2411_03786_b200 as ngs
+    g = np.random.default_rng(52000 + S + Lmax)
+    B, w, topk, k_tab = 10, 4, 5, 6
+    cap = (Lmax + 11) // 4 * 4
+    lens = np.array([Lmax if s % 5 == 0 else int(g.integers(0, Lmax + 1)) for s in range(S)], np.int32)
+    hist = np.full((S, cap), -1, np.int32)
+    for s in range(S):
+        h = g.integers(0, alpha, lens[s])
+        for _ in range(int(lens[s]) // 150):
+            a, b, n = int(g.integers(0, lens[s] - 20)), int(g.integers(0, lens[s] - 20)), int(g.integers(4, 20))
+            h[b:b + n] = h[a:a + n]
+        hist[s, :lens[s]] = h
+    T = np.stack([g.permutation(V)[:k_tab] for _ in range(V)]).astype(np.int32)
+    ext = oracle.extend_table(T, w) if S % 3 == 0 else None
+    ctx.set_model_table(dev_i32(T), dev_i32(ext) if ext is not None else None)
+    fl = flags | (ngs.flag_reserve(3) if S == 600 else 0)
+    want = oracle.draft_batch(hist, lens, qs, topk, B, w, fl, T)
+    for rep in range(2):
+        got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, fl)
+        for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
+            assert np.array_equal(a.cpu().numpy(), b), name
     assert ctx.get_status() == 0
