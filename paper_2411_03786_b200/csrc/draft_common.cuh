@@ -150,8 +150,10 @@ __device__ __forceinline__ void model_chain(const DraftParams& P, int x, int lan
 // comparison chain, per warp iteration one vote; positions go into the warp's queue wq (kMatchQueue
 // ints) and a queue-full is grouped at once, one match per lane, so that the dependent reads a match
 // needs overlap.  No barrier inside: the caller synchronises before (table cleared) and after.
+// Returns how many vectors of the history the calling warp had gone past when it stopped (all of them unless
+// the table overflowed): the caller sizes the next round of passes from it.
 template <int U = 4>  // 128-bit loads a thread keeps in flight
-__device__ __forceinline__ void scan_pass(const DraftParams& P, const int32_t* __restrict__ h, int L, int R, int r,
+__device__ __forceinline__ int scan_pass(const DraftParams& P, const int32_t* __restrict__ h, int L, int R, int r,
                                           int t0, int t1, int t2, int t3, const DraftTable& T, int* wq, int tid, int nthr) {
     const int w = P.w, lane = tid & 31;
     const int n_scan = L - w;  // token index x = p - 1 runs over [0, n_scan)
@@ -183,8 +185,8 @@ __device__ __forceinline__ void scan_pass(const DraftParams& P, const int32_t* _
             }
         }
         const int p = x + 1;
-        uint32_t hc = 0x9E3779B9u;
-        for (int t = 0; t < key_len; ++t) hc = fmix32(hc ^ (uint32_t)h[p + t]) + 0x7F4A7C15u;
+        uint32_t hc = 0x9E3779B9u;  // one multiply-add per token, mixed once per query length below
+        for (int t = 0; t < key_len; ++t) hc = hc * 0x85EBCA6Bu + (uint32_t)h[p + t];
         for (int qi = 0; qi < P.n_q; ++qi) {
             const int q = P.qs[qi];
             if (m < q || L < q + w) continue;
@@ -242,11 +244,15 @@ __device__ __forceinline__ void scan_pass(const DraftParams& P, const int32_t* _
     constexpr uint32_t K = 0x9E3779B1u;
     const uint32_t target = need2 ? (uint32_t)t1 * K + (uint32_t)t0 : (uint32_t)t0;
     const int rot_src = (lane + 31) & 31;
+    int reached = n_vec;
     auto scan_blocks = [&](auto two_tokens) {
         constexpr bool N2 = decltype(two_tokens)::value;
         for (int base = wv * (U * 32); base < n_vec; base += nwarps * (U * 32)) {  // warp-uniform
             // too many groups for one pass: the caller rescans with more passes
-            if (__any_sync(0xffffffffu, *((volatile int*)T.overflow))) break;
+            if (__any_sync(0xffffffffu, *((volatile int*)T.overflow))) {
+                reached = base;
+                break;
+            }
             const int v0 = base + lane;
             int4 vv[U];
             int left[U];
@@ -284,6 +290,17 @@ __device__ __forceinline__ void scan_pass(const DraftParams& P, const int32_t* _
     if (need2) scan_blocks(std::true_type{});
     else scan_blocks(std::false_type{});
     flush_matches();
+    return reached;
+}
+
+// Passes for the next round after a pass of a round of R overflowed when about `reached` of `n_vec` vectors had
+// been scanned: the groups seen so far filled the table, so the whole history needs about n_vec / reached
+// tables' worth per residue class - with a margin, at least twice as many as before, as a power of two.
+__device__ __forceinline__ int next_pass_count(int R, int reached, int n_vec) {
+    const long long est = (long long)R * n_vec * 5 / (4ll * (reached > 0 ? reached : 1)) + 1;
+    int next = 2 * R;
+    while (next < est && next <= kMaxPasses) next *= 2;
+    return next;
 }
 
 // Scratch of the ranking and mixing steps (one per group of threads; see the layouts of the kernels).

@@ -68,7 +68,7 @@ struct StreamMisc {
     int n_cnt[kMaxNQ];
     int cand_off[kMaxNQ + 2];
     int n_surv;
-    int pad_;
+    int reached;
     unsigned long long tau[kMaxNQ];
 };
 
@@ -123,7 +123,9 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) draft_stream_kernel(const D
                         sm->desc[buf].L = L;
                         sm->desc[buf].flags = (r == 0 ? PASS_FIRST : 0) | ((r == R - 1 || gave_up) ? PASS_LAST : 0) | (gave_up ? PASS_GAVE_UP : 0);
                     }
-                    if (scan && !gave_up) scan_pass<STREAM_LOADS>(P, h, L, R, r, t0, t1, t2, t3, T, wq, tid, SWT);
+                    int reached = 0;
+                    if (scan && !gave_up) reached = scan_pass<STREAM_LOADS>(P, h, L, R, r, t0, t1, t2, t3, T, wq, tid, SWT);
+                    if (tid == 0) sm->reached = reached;
                     named_sync(BAR_SCAN, SWT);  // every scanner's matches are in the table
                     overflowed = *((volatile int*)T.overflow) != 0;
                     if (overflowed && tid == 0) sm->desc[buf].flags |= PASS_VOID;  // this pass does not count: more passes follow
@@ -132,7 +134,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) draft_stream_kernel(const D
                     if (gave_up) break;
                 }
                 if (!overflowed || gave_up) break;
-                R *= 2;
+                R = next_pass_count(R, sm->reached, (max(L - P.w, 0) + 3) >> 2);
             }
         }
         // tell the finishers to stop, then wait until they have released the other table too

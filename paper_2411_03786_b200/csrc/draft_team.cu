@@ -58,7 +58,7 @@ struct TeamMisc {
     int tq[kMaxQ];
     int cand_off[kMaxNQ + 2];
     int n_surv;
-    int pad_;
+    int reached;
     unsigned long long tau[kMaxNQ];
 };
 
@@ -168,7 +168,8 @@ __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(cons
                     sm->overflow = 0;
                 }
                 team_sync();
-                scan_pass(P, h, L, R, r, t0, t1, t2, t3, tab, wq, tid, TT);
+                const int reached = scan_pass(P, h, L, R, r, t0, t1, t2, t3, tab, wq, tid, TT);
+                if (tid == 0) sm->reached = reached;
                 team_sync();  // the team's matches are in the table
                 if (*((volatile int*)&sm->overflow)) {
                     overflowed = true;
@@ -177,7 +178,7 @@ __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(cons
                 rank_pass(P, tab, X, tid, TT, team_sync);
             }
             if (!overflowed) break;
-            R *= 2;
+            R = next_pass_count(R, sm->reached, (max(n_scan, 0) + 3) >> 2);
             if (R > kMaxPasses) {
                 gave_up = true;
                 break;
@@ -202,10 +203,11 @@ static int round_up16(int x) { return (x + 15) & ~15; }
 
 int launch_draft_team(spec_ctx* ctx, DraftParams& P, cudaStream_t st) {
     const int sms = ctx->num_sms;
-    // Table: about as many slots as groups are expected (rescans of a staged history are cheap, so the table
-    // may be half of what one pass would need): a query of one token matches up to a tenth of the positions
-    // on natural token statistics, longer queries around one in a hundred.
-    const int expect = P.q_min >= 2 || P.n_q == 0 ? P.cap / 72 : P.cap / 5;
+    // Table: twice as many slots as groups are expected.  A query of one token matches up to a tenth of the
+    // positions on natural token statistics, longer queries around one in a hundred.  (A table that
+    // overflows costs whole rescans - measured on 4096 x 2048 tokens with a one-token query: 128 us with 512
+    // slots, 80 us with 1024 - so the estimate errs on the large side.)
+    const int expect = P.q_min >= 2 || P.n_q == 0 ? P.cap / 72 : P.cap / 4;
     int slots = 256;
     while (slots < expect && slots < 2048) slots <<= 1;
     P.slots = slots;
@@ -220,6 +222,13 @@ int launch_draft_team(spec_ctx* ctx, DraftParams& P, cudaStream_t st) {
     if (const char* ov = getenv("NGRAM_SPEC_TEAM")) {  // tuning builds only: warps per team
         const int t = atoi(ov);
         if (t == 1 || t == 2 || t == 4 || t == 8 || t == 16) T = t;
+    }
+    if (const char* ov = getenv("NGRAM_SPEC_TEAM_SLOTS")) {  // ... and table slots
+        const int t = atoi(ov);
+        if (t >= 64 && t <= 4096 && (t & (t - 1)) == 0) {
+            P.slots = t;
+            P.max_groups = t / 2;
+        }
     }
 #endif
     TeamLayout Y{};
@@ -255,6 +264,7 @@ int launch_draft_team(spec_ctx* ctx, DraftParams& P, cudaStream_t st) {
         if (teams > TEAM_MAX_WARPS / T) teams = TEAM_MAX_WARPS / T;
         if (T > 1 && teams > 8) teams = 8;
         Y.teams = teams;
+        if (teams == 1 && T < 16) continue;    // room for one sequence only: all 16 warps work on it
         if (teams * T >= 8 || T == 16) break;  // at least eight warps per CTA, or the largest team
     }
     if (Y.teams < 1) return kDraftNoFit;
