@@ -30,7 +30,10 @@ namespace ngs {
 constexpr int STREAM_SCAN_WARPS = 24, STREAM_POST_WARPS = 7;
 constexpr int SWT = STREAM_SCAN_WARPS * 32, PWT = STREAM_POST_WARPS * 32;
 constexpr int STREAM_THREADS = SWT + PWT + 32;
-constexpr int STREAM_LOADS = 6;          // 128-bit loads a scanner thread keeps in flight
+#ifndef NGRAM_STREAM_LOADS
+#define NGRAM_STREAM_LOADS 6
+#endif
+constexpr int STREAM_LOADS = NGRAM_STREAM_LOADS;  // 128-bit loads a scanner thread keeps in flight
 // named barriers (barrier 0 is the CTA's); + b = table, + k = descriptor slot
 constexpr int BAR_FULL = 1;     // table b complete               (scanners arrive, finishers wait)
 constexpr int BAR_EMPTY = 3;    // table b cleared and free       (finishers arrive, scanners wait)
