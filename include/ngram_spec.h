@@ -62,7 +62,8 @@ enum {
     SPEC_STATUS_TOKEN_RANGE = 1, /* a draft row (context or model) held a token outside [0, V): the row was dropped */
     SPEC_STATUS_CAPACITY = 2,    /* len > cap, or a commit did not fit: that sequence was skipped */
     SPEC_STATUS_TIMEOUT = 4,     /* a bounded device-side wait expired; results of that call are invalid */
-    SPEC_STATUS_GROUPS = 8       /* more distinct continuations than the drafter can group exactly */
+    SPEC_STATUS_GROUPS = 8,      /* more distinct continuations than the drafter can group exactly */
+    SPEC_STATUS_INDEX = 16       /* a context index could not take a window: that sequence is drafted by scanning until the index is rebuilt */
 };
 
 enum { SPEC_F32 = 0, SPEC_BF16 = 1 };
@@ -157,6 +158,37 @@ int spec_set_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, con
 int draft_context_ngrams(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap,
                          const int* qs, int n_q, int topk, int B, int w, int flags, int32_t* d_drafts,
                          int32_t* d_ndrafts, int32_t* d_src, int32_t* d_counts, void* stream);
+
+/*
+ * Incremental context index (Section 4.2 defines the context N-gram as a search of the whole context at
+ * every step; Section 3 wants drafting to cost next to nothing).  The index keeps, per sequence and query
+ * length, what that search would find - every group (q-gram, w-token continuation) with its count and
+ * latest occurrence - in a hash table in caller-owned device memory.  accept_and_commit_indexed adds the
+ * windows that a step's committed tokens completed; draft_context_ngrams_indexed looks the current q-grams
+ * up instead of reading the history.  The drafts are those of draft_context_ngrams, bit for bit: whenever
+ * the index cannot answer for a sequence (its length is not the one the index was last updated to, a table
+ * ran out of probes [SPEC_STATUS_INDEX], or the lookup met more than 2048 groups) that sequence is drafted by
+ * scanning inside the same call.
+ *   spec_context_index_bytes   size of the index for S sequences of capacity cap and n_q query lengths
+ *                              (two 16-byte slots per token of capacity and query length).
+ *   spec_context_index_build   builds the index of the current histories (one-off; also the way to repair
+ *                              an index that fell out of step) and registers it with the context.  qs / n_q:
+ *                              the query lengths to index; w: draft width; flags: SPEC_FLAG_KEY_NEXT_TOKEN or 0.
+ *   draft_context_ngrams_indexed  as draft_context_ngrams; d_index must be the registered index, w and the
+ *                              key flag those it was built with, every q one of its query lengths.
+ *   accept_and_commit_indexed  as accept_and_commit, followed by the index update.  Commits made by any
+ *                              other call leave the index out of step (detected by the length).
+ * The index assumes that the tokens already in a history never change.
+ */
+size_t spec_context_index_bytes(int S, int cap, int n_q);
+int spec_context_index_build(spec_ctx* ctx, void* d_index, const int32_t* d_hist, const int32_t* d_len, int S, int cap,
+                             const int* qs, int n_q, int w, int flags, void* stream);
+int draft_context_ngrams_indexed(spec_ctx* ctx, const void* d_index, const int32_t* d_hist, const int32_t* d_len, int S, int cap,
+                                 const int* qs, int n_q, int topk, int B, int w, int flags, int32_t* d_drafts,
+                                 int32_t* d_ndrafts, int32_t* d_src, int32_t* d_counts, void* stream);
+int accept_and_commit_indexed(spec_ctx* ctx, void* d_index, const int32_t* d_drafts, const int32_t* d_ndrafts,
+                              const int32_t* d_argmax, int S, int B, int w, int32_t* d_hist, int32_t* d_len, int cap,
+                              int32_t* d_acc_len, int32_t* d_best_row, int32_t* d_committed, void* stream);
 
 /*
  * Verification head (Section 3: the model call on a (k, w+1) block; here its LM-head part).

@@ -10,7 +10,7 @@ import torch
 from .build import LIB, build_library
 
 FLAG_DEDUP, FLAG_MODEL_FILL, FLAG_KEY_NEXT_TOKEN = 1, 2, 4
-STATUS_TOKEN_RANGE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_GROUPS = 1, 2, 4, 8
+STATUS_TOKEN_RANGE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_GROUPS, STATUS_INDEX = 1, 2, 4, 8, 16
 SPEC_F32, SPEC_BF16 = 0, 1
 
 _HEADER = os.path.join(os.path.dirname(os.path.abspath(__file__)), "..", "include", "ngram_spec.h")
@@ -70,6 +70,13 @@ def load_library(build: bool = True) -> C.CDLL:
     lib.build_model_ngram_table_rows.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, i32p, fp, vp]
     lib.spec_extend_model_table.argtypes = [vp, i32p, C.c_int, C.c_int, i32p, vp]
     lib.spec_debug_expire_wait.argtypes = [vp, C.c_ulonglong, C.c_int, vp]
+    lib.spec_context_index_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+    lib.spec_context_index_bytes.restype = C.c_size_t
+    lib.spec_context_index_build.argtypes = [vp, vp, i32p, i32p, C.c_int, C.c_int, ip, C.c_int, C.c_int, C.c_int, vp]
+    lib.draft_context_ngrams_indexed.argtypes = [vp, vp, i32p, i32p, C.c_int, C.c_int, ip, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                 C.c_int, i32p, i32p, i32p, i32p, vp]
+    lib.accept_and_commit_indexed.argtypes = [vp, vp, i32p, i32p, i32p, C.c_int, C.c_int, C.c_int, i32p, i32p, C.c_int, i32p,
+                                              i32p, i32p, vp]
     lib.spec_launch_count.argtypes = [vp]
     lib.spec_launch_count.restype = C.c_longlong
     _lib = lib
@@ -193,6 +200,47 @@ class SpecContext:
                                                    qs_arr, len(qs), topk, B, w, flags, _ptr(drafts), _ptr(nd),
                                                    _ptr(src), _ptr(counts), _stream()), "draft_context_ngrams")
         return drafts, nd, src, counts
+
+    def context_index_build(self, hist: torch.Tensor, lens: torch.Tensor, qs, w: int, flags: int = 0, index: torch.Tensor | None = None):
+        """Builds (and registers) the incremental context index of the current histories; returns the index buffer."""
+        S, cap = int(hist.shape[0]), int(hist.shape[1])
+        need = int(self._lib.spec_context_index_bytes(S, cap, len(qs)))
+        if index is None:
+            index = torch.empty(need, dtype=torch.uint8, device=hist.device)
+        assert index.numel() >= need
+        qs_arr = (C.c_int * max(1, len(qs)))(*[int(q) for q in qs])
+        self._check(self._lib.spec_context_index_build(self._h, _ptr(index), _ptr(hist, torch.int32), _ptr(lens, torch.int32), S, cap,
+                                                       qs_arr, len(qs), w, flags, _stream()), "spec_context_index_build")
+        self._keep_index = index
+        return index
+
+    def draft_context_ngrams_indexed(self, index: torch.Tensor, hist: torch.Tensor, lens: torch.Tensor, qs, topk: int, B: int, w: int,
+                                     flags: int = FLAG_DEDUP | FLAG_MODEL_FILL, out=None):
+        S, cap = int(hist.shape[0]), int(hist.shape[1])
+        dev = hist.device
+        if out is None:
+            out = (torch.empty((S, B, w), dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+                   torch.empty((S, B), dtype=torch.int32, device=dev), torch.empty((S, B), dtype=torch.int32, device=dev))
+        drafts, nd, src, counts = out
+        qs_arr = (C.c_int * max(1, len(qs)))(*[int(q) for q in qs])
+        self._check(self._lib.draft_context_ngrams_indexed(self._h, _ptr(index), _ptr(hist, torch.int32), _ptr(lens, torch.int32), S, cap,
+                                                           qs_arr, len(qs), topk, B, w, flags, _ptr(drafts), _ptr(nd),
+                                                           _ptr(src), _ptr(counts), _stream()), "draft_context_ngrams_indexed")
+        return drafts, nd, src, counts
+
+    def accept_and_commit_indexed(self, index: torch.Tensor, drafts, n_drafts, argmax, hist, lens, out=None):
+        S, B, w = (int(x) for x in drafts.shape)
+        cap = int(hist.shape[1])
+        dev = hist.device
+        if out is None:
+            out = (torch.empty(S, dtype=torch.int32, device=dev), torch.empty(S, dtype=torch.int32, device=dev),
+                   torch.empty((S, w + 1), dtype=torch.int32, device=dev))
+        acc, best, com = out
+        self._check(self._lib.accept_and_commit_indexed(self._h, _ptr(index), _ptr(drafts, torch.int32), _ptr(n_drafts, torch.int32),
+                                                        _ptr(argmax, torch.int32), S, B, w, _ptr(hist, torch.int32),
+                                                        _ptr(lens, torch.int32), cap, _ptr(acc), _ptr(best), _ptr(com),
+                                                        _stream()), "accept_and_commit_indexed")
+        return acc, best, com
 
     def verify_lmhead_argmax(self, hidden: torch.Tensor, out=None, with_max: bool = False):
         M = int(hidden.shape[0])

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libngram_spec.so")
-SOURCES = ["api.cu", "accept.cu", "draft.cu", "draft_team.cu", "draft_stream.cu", "head_gemm.cu"]
+SOURCES = ["api.cu", "accept.cu", "draft.cu", "draft_team.cu", "draft_stream.cu", "ctx_index.cu", "head_gemm.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "-cudart", "static"]
 

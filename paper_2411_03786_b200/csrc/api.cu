@@ -8,6 +8,7 @@
 
 #include "accept.cuh"
 #include "common.cuh"
+#include "draft_common.cuh"
 
 // Error text of calls that have no context to keep it in: one buffer per host thread.
 static thread_local char g_err[256] = "";
@@ -270,6 +271,62 @@ int draft_context_ngrams(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_
     cudaSetDevice(ctx->device);
     return launch_draft(ctx, d_hist, d_len, S, cap, qs, n_q, topk, B, w, flags, d_drafts, d_ndrafts, d_src, d_counts,
                         (cudaStream_t)stream);
+}
+
+size_t spec_context_index_bytes(int S, int cap, int n_q) {
+    if (S < 0 || cap <= 0 || n_q < 1 || n_q > kMaxNQ) return 0;
+    return context_index_bytes(S, cap, n_q);
+}
+
+int spec_context_index_build(spec_ctx* ctx, void* d_index, const int32_t* d_hist, const int32_t* d_len, int S, int cap,
+                             const int* qs, int n_q, int w, int flags, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "spec_context_index_build: ctx is NULL");
+    if (!d_index || !d_hist || !d_len || !qs) return fail(ctx, SPEC_ERR_ARG, "spec_context_index_build: NULL pointer");
+    if (!aligned16(d_index) || !aligned16(d_hist)) return fail(ctx, SPEC_ERR_ARG, "spec_context_index_build: d_index and d_hist must be 16-byte aligned");
+    if (S < 1 || cap <= 0 || cap % 4 != 0 || cap >= (1 << 28)) return fail(ctx, SPEC_ERR_ARG, "spec_context_index_build: need S >= 1, 0 < cap < 2^28, cap %% 4 == 0");
+    if (n_q < 1 || n_q > kMaxNQ || w < 1 || w > kMaxW) return fail(ctx, SPEC_ERR_ARG, "spec_context_index_build: need 1<=n_q<=%d, 1<=w<=%d", kMaxNQ, kMaxW);
+    for (int i = 0; i < n_q; ++i) {
+        if (qs[i] < 1 || qs[i] > kMaxQ) return fail(ctx, SPEC_ERR_ARG, "spec_context_index_build: q must be in [1, %d]", kMaxQ);
+        for (int j = 0; j < i; ++j)
+            if (qs[j] == qs[i]) return fail(ctx, SPEC_ERR_ARG, "spec_context_index_build: query lengths must be distinct");
+    }
+    if (flags & ~SPEC_FLAG_KEY_NEXT_TOKEN) return fail(ctx, SPEC_ERR_ARG, "spec_context_index_build: flags may only hold SPEC_FLAG_KEY_NEXT_TOKEN");
+    cudaSetDevice(ctx->device);
+    return launch_index_build(ctx, d_index, d_hist, d_len, S, cap, qs, n_q, w, (flags & SPEC_FLAG_KEY_NEXT_TOKEN) ? 1 : w, (cudaStream_t)stream);
+}
+
+int draft_context_ngrams_indexed(spec_ctx* ctx, const void* d_index, const int32_t* d_hist, const int32_t* d_len, int S, int cap,
+                                 const int* qs, int n_q, int topk, int B, int w, int flags, int32_t* d_drafts,
+                                 int32_t* d_ndrafts, int32_t* d_src, int32_t* d_counts, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "draft_context_ngrams_indexed: ctx is NULL");
+    if (!d_hist || !d_len || !d_drafts || !d_ndrafts) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: NULL pointer");
+    if (B < 1 || B > kMaxB || w < 1 || w > kMaxW) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: need 1<=B<=%d, 1<=w<=%d", kMaxB, kMaxW);
+    if (n_q < 0 || n_q > kMaxNQ || (n_q > 0 && !qs)) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: need 0<=n_q<=%d", kMaxNQ);
+    if (topk < 1 || topk > B) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: need 1 <= topk <= B");
+    const spec_ctx::IndexMeta& m = ctx->index;
+    if (!d_index || d_index != m.ptr) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: d_index is not the index registered by spec_context_index_build");
+    if (S != m.S || cap != m.cap || w != m.w || ((flags & SPEC_FLAG_KEY_NEXT_TOKEN) ? 1 : w) != m.key_len)
+        return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: S, cap, w and the key flag must be those the index was built with");
+    if ((flags & SPEC_FLAG_MODEL_FILL) && !ctx->tab_idx)
+        return fail(ctx, SPEC_ERR_NOT_BUILT, "draft_context_ngrams_indexed: model fill needs build_model_ngram_tables first");
+    cudaSetDevice(ctx->device);
+    DraftParams P = make_draft_params(ctx, d_hist, d_len, S, cap, qs, n_q, topk, B, w, flags, d_drafts, d_ndrafts, d_src, d_counts);
+    return launch_draft_indexed(ctx, P, (cudaStream_t)stream);
+}
+
+int accept_and_commit_indexed(spec_ctx* ctx, void* d_index, const int32_t* d_drafts, const int32_t* d_ndrafts,
+                              const int32_t* d_argmax, int S, int B, int w, int32_t* d_hist, int32_t* d_len, int cap,
+                              int32_t* d_acc_len, int32_t* d_best_row, int32_t* d_committed, void* stream) {
+    if (!ctx) return fail(nullptr, SPEC_ERR_ARG, "accept_and_commit_indexed: ctx is NULL");
+    if (!d_drafts || !d_ndrafts || !d_argmax || !d_hist || !d_len || !d_acc_len || !d_best_row || !d_committed)
+        return fail(ctx, SPEC_ERR_ARG, "accept_and_commit_indexed: NULL pointer");
+    if (B < 1 || B > kMaxB || w < 1 || w > kMaxW) return fail(ctx, SPEC_ERR_ARG, "accept_and_commit_indexed: need 1<=B<=%d, 1<=w<=%d", kMaxB, kMaxW);
+    const spec_ctx::IndexMeta& m = ctx->index;
+    if (!d_index || d_index != m.ptr) return fail(ctx, SPEC_ERR_ARG, "accept_and_commit_indexed: d_index is not the index registered by spec_context_index_build");
+    if (S != m.S || cap != m.cap || w != m.w) return fail(ctx, SPEC_ERR_ARG, "accept_and_commit_indexed: S, cap and w must be those the index was built with");
+    cudaSetDevice(ctx->device);
+    const AcceptArgs q{d_drafts, d_ndrafts, d_argmax, S, B, w, d_hist, d_len, cap, d_acc_len, d_best_row, d_committed, ctx->d_status};
+    return launch_accept_indexed(ctx, q, (cudaStream_t)stream);
 }
 
 int verify_lmhead_argmax(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax, float* d_max, void* stream) {

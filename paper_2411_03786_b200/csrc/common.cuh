@@ -72,6 +72,12 @@ struct spec_ctx {
         CUtensorMap tm;
     } a_maps[4];
     int a_map_next = 0;
+    // the incremental context index registered with this context (caller-owned memory)
+    struct IndexMeta {
+        void* ptr = nullptr;
+        int S = 0, cap = 0, n_q = 0, w = 0, key_len = 0, slots = 0;
+        int qs[4] = {0, 0, 0, 0};
+    } index;
     void* d_centred = nullptr;  // unigram scratch: bf16 [V, d] output embeddings minus their mean
     float* d_colsum = nullptr;  // unigram scratch: [64 + 1, d] partial column sums and the mean
     long long launches = 0;
@@ -158,6 +164,11 @@ int launch_extend_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, int 
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st);
 int launch_unigram(spec_ctx* ctx, int k_uni, int32_t* d_uni_idx, float* d_dist2, cudaStream_t st);
 int launch_wait_probe(spec_ctx* ctx, unsigned long long limit_ns, int mark_incomplete, cudaStream_t st);
+// ctx_index.cu
+size_t context_index_bytes(int S, int cap, int n_q);
+int launch_index_build(spec_ctx* ctx, void* d_index, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs,
+                       int n_q, int w, int key_len, cudaStream_t st);
+int launch_accept_indexed(spec_ctx* ctx, const AcceptArgs& a, cudaStream_t st);
 // draft.cu / accept.cu
 int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
                  int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,

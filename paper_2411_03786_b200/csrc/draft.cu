@@ -475,9 +475,9 @@ __global__ void __launch_bounds__(1024, 1) draft_kernel(const DraftParams P) {
     if (tid == 0) P.ndrafts[s] = n;
 }
 
-int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
-                 int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,
-                 int32_t* d_counts, cudaStream_t st) {
+DraftParams make_draft_params(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
+                              int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,
+                              int32_t* d_counts) {
     DraftParams P;
     P.hist = d_hist;
     P.len = d_len;
@@ -505,6 +505,17 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     P.src = d_src;
     P.counts = d_counts;
     P.status = ctx->d_status;
+    P.slots = 0;
+    P.max_groups = 0;
+    P.stage_hist = 0;
+    P.hist_off = 0;
+    return P;
+}
+
+int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
+                 int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,
+                 int32_t* d_counts, cudaStream_t st) {
+    DraftParams P = make_draft_params(ctx, d_hist, d_len, S, cap, qs, n_q, topk, B, w, flags, d_drafts, d_ndrafts, d_src, d_counts);
     int slots = 1024;  // at most slots / 2 distinct continuations are grouped in one pass
     while (slots < cap / 2 && slots < 8192) slots <<= 1;
     int threads = cap >= 16384 ? 1024 : (cap >= 2048 ? 256 : 128);

@@ -336,29 +336,12 @@ struct DraftScratch {
 // among themselves is their rank among all.  The table's memory holds the survivors (the table itself is no
 // longer needed once the keys are built).
 constexpr int kRankDirect = 96;  // up to this many keys are ranked directly
+// Ranks the n_keys keys in X.gkey (rank_acc zeroed, n_cnt zeroed, *n_surv = 0, all before a barrier); `skey` is
+// room for n_keys more keys.  Writes run_key / n_run.  Ends with a barrier.
 template <class Sync>
-__device__ __forceinline__ void rank_pass(const DraftParams& P, const DraftTable& T, const DraftScratch& X, int tid, int nthr,
-                                          Sync&& sync) {
+__device__ __forceinline__ void rank_keys(const DraftParams& P, int n_keys, unsigned long long* skey, const DraftScratch& X, int tid,
+                                          int nthr, Sync&& sync) {
     const int topk = P.topk, lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
-    const int n_groups = *T.n_groups;
-    int n_old = 0;
-    for (int qi = 0; qi < P.n_q; ++qi) n_old += X.n_run[qi];
-    const int n_keys = n_groups + n_old;
-    for (int g = tid; g < n_groups; g += nthr) {
-        const int slot = T.grp_slot[g];
-        const unsigned long long qi = (unsigned long long)(T.rep[slot] >> 28);
-        X.gkey[g] = (qi << 60) | ((unsigned long long)(uint32_t)T.cnt[slot] << 32) | (uint32_t)T.last[slot];
-        X.rank_acc[g] = 0;
-    }
-    for (int j = tid; j < n_old; j += nthr) {
-        int qi = 0, o = j;
-        while (o >= X.n_run[qi]) o -= X.n_run[qi++];
-        X.gkey[n_groups + j] = ((unsigned long long)qi << 60) | X.run_key[qi * topk + o];
-        X.rank_acc[n_groups + j] = 0;
-    }
-    if (tid < kMaxNQ) X.n_cnt[tid] = 0;
-    if (tid == 0) *X.n_surv = 0;
-    sync();
     const unsigned long long* keys = X.gkey;
     int m = n_keys;
     if (n_keys > kRankDirect) {
@@ -385,7 +368,6 @@ __device__ __forceinline__ void rank_pass(const DraftParams& P, const DraftTable
             if (lane == 0) X.tau[qi] = tau;
         }
         sync();
-        unsigned long long* skey = reinterpret_cast<unsigned long long*>(T.rep);
         for (int g = tid; g < n_keys; g += nthr) {
             const unsigned long long k = X.gkey[g];
             if (k >= X.tau[(int)(k >> 60)]) {
@@ -432,6 +414,34 @@ __device__ __forceinline__ void rank_pass(const DraftParams& P, const DraftTable
     sync();
     if (tid < kMaxNQ) X.n_run[tid] = X.n_cnt[tid];
     sync();
+}
+
+// A finished pass: the keys of table T's groups and of the winners so far, then rank_keys.  The table's
+// memory holds the survivors (the table itself is no longer needed once the keys are built).
+template <class Sync>
+__device__ __forceinline__ void rank_pass(const DraftParams& P, const DraftTable& T, const DraftScratch& X, int tid, int nthr,
+                                          Sync&& sync) {
+    const int topk = P.topk;
+    const int n_groups = *T.n_groups;
+    int n_old = 0;
+    for (int qi = 0; qi < P.n_q; ++qi) n_old += X.n_run[qi];
+    const int n_keys = n_groups + n_old;
+    for (int g = tid; g < n_groups; g += nthr) {
+        const int slot = T.grp_slot[g];
+        const unsigned long long qi = (unsigned long long)(T.rep[slot] >> 28);
+        X.gkey[g] = (qi << 60) | ((unsigned long long)(uint32_t)T.cnt[slot] << 32) | (uint32_t)T.last[slot];
+        X.rank_acc[g] = 0;
+    }
+    for (int j = tid; j < n_old; j += nthr) {
+        int qi = 0, o = j;
+        while (o >= X.n_run[qi]) o -= X.n_run[qi++];
+        X.gkey[n_groups + j] = ((unsigned long long)qi << 60) | X.run_key[qi * topk + o];
+        X.rank_acc[n_groups + j] = 0;
+    }
+    if (tid < kMaxNQ) X.n_cnt[tid] = 0;
+    if (tid == 0) *X.n_surv = 0;
+    sync();
+    rank_keys(P, n_keys, reinterpret_cast<unsigned long long*>(T.rep), X, tid, nthr, sync);
 }
 
 // Mixed allocation of sequence s: context rows in query order, then model rows by rank; duplicates dropped;
@@ -564,6 +574,13 @@ __device__ __forceinline__ void mix_and_emit(const DraftParams& P, int s, const 
     if (tid == 0) P.ndrafts[s] = n;
     sync();
 }
+
+// draft.cu
+DraftParams make_draft_params(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int S, int cap, const int* qs, int n_q,
+                              int topk, int B, int w, int flags, int32_t* d_drafts, int32_t* d_ndrafts, int32_t* d_src,
+                              int32_t* d_counts);
+// ctx_index.cu
+int launch_draft_indexed(spec_ctx* ctx, DraftParams& P, cudaStream_t st);
 
 // draft_team.cu / draft_stream.cu
 constexpr int kDraftNoFit = 1;  // launch_draft_team: the staged layout does not fit (nothing was launched)
