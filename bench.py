@@ -202,8 +202,13 @@ def scaled_streams(ctx, torch, dev, c, pk):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / reps
 
-    for S, L, qs, reps in ((4096, 2048, (3, 2, 1), 20), (512, 131072, (3, 2), 5)):   # shaped like C3 / C5
-        base, lens_b, _ = synth.zipf_histories(32, L, c["V"], c["zipf"], 0.3, seed=77, cap=L + 64, name="scaled")
+    # shaped like C3 (V = 32000, Zipf 1.1) and like C5 (V = 128256, Zipf 1.05); the third entry keeps the 32000-token
+    # vocabulary on the long histories (more matches per sequence)
+    for S, L, qs, reps, Vz, zz, tag in ((4096, 2048, (3, 2, 1), 20, 32000, 1.1, ""), (512, 131072, (3, 2), 5, 128256, 1.05, ""),
+                                        (512, 131072, (3, 2), 5, 32000, 1.1, "_V32000")):
+        if ctx.V < Vz:
+            continue
+        base, lens_b, _ = synth.zipf_histories(32, L, Vz, zz, 0.3, seed=77, cap=L + 64, name="scaled")
         hist = torch.from_numpy(np.tile(base, (S // 32, 1))).to(dev)
         lens = torch.from_numpy(np.tile(lens_b, S // 32)).to(dev)
         B, w, topk = 16, 8, 4
@@ -211,7 +216,12 @@ def scaled_streams(ctx, torch, dev, c, pk):
                 torch.empty((S, B), dtype=torch.int32, device=dev), torch.empty((S, B), dtype=torch.int32, device=dev))
         ms = timed(lambda: ctx.draft_context_ngrams(hist, lens, qs, topk, B, w, out=bufs), reps)
         by = 4.0 * S * L + 4.0 * S * B * (w + 2) + 8.0 * S
-        out[f"draft_S{S}_L{L}"] = {"qs": list(qs), "ms": ms, "GB/s": by / ms / 1e6, "frac_of_hbm": by / ms / 1e6 / pk["hbm"],
+        ix_ms = None
+        if L >= 131072 and not tag:   # the same batch drafted from the incremental context index (built once, outside the timing)
+            index = ctx.context_index_build(hist, lens, qs, w)
+            ix_ms = timed(lambda: ctx.draft_context_ngrams_indexed(index, hist, lens, qs, topk, B, w, out=bufs), reps)
+            del index
+        out[f"draft_S{S}_L{L}{tag}"] = {"qs": list(qs), "vocabulary": Vz, "zipf": zz, "ms": ms, "ms_from_context_index": ix_ms, "GB/s": by / ms / 1e6, "frac_of_hbm": by / ms / 1e6 / pk["hbm"],
                                    "frac_of_nominal_hbm": by / ms / 1e6 / NOMINAL["hbm_gbs"], "bytes": by,
                                    "l2": "larger than L2" if by > 126e6 else "L2-resident"}
         del hist, lens, bufs
@@ -505,9 +515,77 @@ def measure_config(torch, ngs, c, head, dev, pk, args, rank, dist, headline):
            "roofline": roof, "copied_fraction": copied}
     if fp8:
         rec["fp8_verify"] = fp8
+    if headline or c["name"] in ("C2", "C3"):
+        rec["context_index"] = index_comparison(torch, c, head, dict(hist=hist, lens0=lens0, out_v=out_v, out_d=out_d, out_a=out_a, side=side), dev)
     extra = dict(hist_h=hist_h, lens_h=lens_h, H_bits=H_bits, hist=hist, lens0=lens0, dH=dH, out_d=out_d, out_v=out_v, out_a=out_a,
                  acc_tokens=acc_tokens, side=side, clocks=clocks, n_blocks=len(blocks), n_fblocks=len(fblocks), K=K, barrier=barrier)
     return rec, extra
+
+
+def index_comparison(torch, c, head, x, dev):
+    """Drafting + acceptance of consecutive decode steps with the history scanned at every step, and with the
+    incremental context index (looked up by the draft, updated by the commit).  Each variant is one CUDA graph of
+    `n` steps on its own copy of the histories (the steps really advance: a token or more is committed per step)."""
+    ctx = head.ctx
+    S, B, w, M = c["S"], c["B"], c["w"], c["M"]
+    n = 24
+    cap2 = (c["L"] + n * (w + 1) + 8 + 3) // 4 * 4
+    hist0 = torch.full((S, cap2), -1, dtype=torch.int32, device=dev)
+    hist0[:, :x["hist"].shape[1]] = x["hist"]
+    lens0 = x["lens0"].clone()
+    P = x["out_v"][0].view(S, B, w + 1).clone()          # the planted step's predictions, reused at every step
+    out_d = tuple(torch.empty_like(t) for t in x["out_d"])
+    out_a = tuple(torch.empty_like(t) for t in x["out_a"])
+    res = {"steps_per_graph": n, "note": "draft + accept per step, steps advance the history; planted predictions of the first step reused"}
+    side = x["side"]
+    for kind in ("scan", "index"):
+        hist, lens = hist0.clone(), lens0.clone()
+        index = ctx.context_index_build(hist, lens, c["qs"], w) if kind == "index" else None
+
+        def steps():
+            for _ in range(n):
+                if kind == "index":
+                    ctx.draft_context_ngrams_indexed(index, hist, lens, c["qs"], c["topk"], B, w, out=out_d)
+                    ctx.accept_and_commit_indexed(index, out_d[0], out_d[1], P, hist, lens, out=out_a)
+                else:
+                    ctx.draft_context_ngrams(hist, lens, c["qs"], c["topk"], B, w, out=out_d)
+                    ctx.accept_and_commit(out_d[0], out_d[1], P, hist, lens, out=out_a)
+
+        def reset():
+            hist.copy_(hist0)
+            lens.copy_(lens0)
+            if kind == "index":
+                ctx.context_index_build(hist, lens, c["qs"], w, index=index)
+
+        with torch.cuda.stream(side):
+            steps()
+        torch.cuda.synchronize()
+        reset()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            steps()
+        ts = []
+        for _ in range(5):
+            reset()
+            torch.cuda.synchronize()
+            a, b = ev(torch), ev(torch)
+            a.record()
+            g.replay()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / n)
+        res[kind] = {"us_per_step": statistics.median(ts) * 1e3, "tokens_committed": int((lens - lens0).sum().item())}
+        if kind == "index":
+            t0 = ev(torch), ev(torch)
+            t0[0].record()
+            ctx.context_index_build(hist, lens, c["qs"], w, index=index)
+            t0[1].record()
+            torch.cuda.synchronize()
+            res["index"]["build_ms"] = t0[0].elapsed_time(t0[1])
+            res["index"]["bytes"] = int(index.numel())
+    assert res["scan"]["tokens_committed"] == res["index"]["tokens_committed"], "the two variants decoded differently"
+    assert ctx.get_status() == 0
+    return res
 
 
 def workload_string(c):
@@ -807,6 +885,8 @@ def main():
                 "peaks": {"measured": pk, "nominal": NOMINAL}}
         if "fp8_verify" in head_rec:
             line["fp8_verify"] = head_rec["fp8_verify"]
+        if "context_index" in head_rec:
+            line["context_index"] = head_rec["context_index"]
         if per_config:
             line["per_config"] = per_config
         if scaled:

@@ -170,7 +170,7 @@ int draft_context_ngrams(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_
  * ran out of probes [SPEC_STATUS_INDEX], or the lookup met more than 2048 groups) that sequence is drafted by
  * scanning inside the same call.
  *   spec_context_index_bytes   size of the index for S sequences of capacity cap and n_q query lengths
- *                              (two 16-byte slots per token of capacity and query length).
+ *                              (1.5 to 3 16-byte slots per token of capacity and query length).
  *   spec_context_index_build   builds the index of the current histories (one-off; also the way to repair
  *                              an index that fell out of step) and registers it with the context.  qs / n_q:
  *                              the query lengths to index; w: draft width; flags: SPEC_FLAG_KEY_NEXT_TOKEN or 0.

@@ -16,7 +16,7 @@
 //           tag = 16 bits of a second q-gram hash | 16 bits of a continuation hash (a filter: equality is
 //           always confirmed on the tokens)
 //   count = windows in the group,  last = latest continuation start of the group.
-// A table has at least twice as many slots as the history capacity, so it never fills.
+// A table has at least 1.5 times as many slots as the history capacity, so it never fills.
 #include "accept.cuh"
 #include "draft_common.cuh"
 
@@ -42,9 +42,9 @@ struct IndexView {
 };
 
 static size_t index_state_bytes(int S) { return ((size_t)S * 8 + 15) & ~size_t(15); }
-static int index_slots(int cap) {
+static int index_slots(int cap) {  // a power of two at least 1.5 times the capacity: never more than two thirds full
     int s = 64;
-    while (s < 2 * cap) s <<= 1;
+    while (2 * s < 3 * cap) s <<= 1;
     return s;
 }
 
@@ -63,18 +63,49 @@ static IndexView make_view(const spec_ctx::IndexMeta& m) {
     return v;
 }
 
-__device__ __forceinline__ uint32_t hash_tokens(const int32_t* t, int n, uint32_t seed) {
+// Hash of n tokens held in registers (n <= N).
+template <int N>
+__device__ __forceinline__ uint32_t hash_tokens(const int (&t)[N], int n, uint32_t seed) {
     uint32_t hsh = seed;
-    for (int i = 0; i < n; ++i) hsh = hsh * 0x85EBCA6Bu + (uint32_t)t[i];
+#pragma unroll
+    for (int i = 0; i < N; ++i)
+        if (i < n) hsh = hsh * 0x85EBCA6Bu + (uint32_t)t[i];
     return fmix32(hsh);
 }
 
-// Adds the window whose continuation starts at p (q-gram hist[p - q .. p), p >= q, p + w <= length) to table
-// `tbl`.  Safe against concurrent inserts into the same table.  Returns false if the probe run never ended.
-__device__ __forceinline__ bool index_insert(IndexEntry* tbl, int slots, const int32_t* h, int p, int q, int key_len) {
-    const uint32_t qh = hash_tokens(h + p - q, q, 0x9E3779B9u);
-    const uint32_t ch = hash_tokens(h + p, key_len, 0x7F4A7C15u);
-    const uint32_t tag = (fmix32(qh + 0x632BE5ABu) & 0xFFFF0000u) | (ch >> 16);
+// A window in registers: qg[t] = the q-gram's token t + 1 places before the continuation start, ct[t] = the
+// continuation's token t.  All loads are issued before the first use (one memory latency, not q + w of them).
+struct Window {
+    int qg[kMaxQ];
+    int ct[kMaxW];
+};
+__device__ __forceinline__ Window load_window(const int32_t* h, int p, int q, int key_len) {
+    Window wv;
+#pragma unroll
+    for (int t = 0; t < kMaxQ; ++t) wv.qg[t] = t < q ? h[p - 1 - t] : 0;
+#pragma unroll
+    for (int t = 0; t < kMaxW; ++t) wv.ct[t] = t < key_len ? h[p + t] : 0;
+    return wv;
+}
+__device__ __forceinline__ bool same_window(const Window& a, const int32_t* h, int rp, int q, int key_len) {
+    int diff = 0;
+#pragma unroll
+    for (int t = 0; t < kMaxQ; ++t)
+        if (t < q) diff |= h[rp - 1 - t] ^ a.qg[t];
+#pragma unroll
+    for (int t = 0; t < kMaxW; ++t)
+        if (t < key_len) diff |= h[rp + t] ^ a.ct[t];
+    return diff == 0;
+}
+__device__ __forceinline__ uint32_t qgram_hash(const int (&qg)[kMaxQ], int q) { return hash_tokens(qg, q, 0x9E3779B9u); }
+__device__ __forceinline__ uint32_t qgram_tag16(uint32_t qh) { return fmix32(qh + 0x632BE5ABu) >> 16; }
+
+// Adds the window wv whose continuation starts at p (q-gram hist[p - q .. p), p >= q, p + w <= length) to
+// table `tbl`.  Safe against concurrent inserts into the same table.  Returns false if the probe run never ended.
+__device__ __forceinline__ bool index_insert(IndexEntry* tbl, int slots, const int32_t* h, const Window& wv, int p, int q, int key_len) {
+    const uint32_t qh = qgram_hash(wv.qg, q);
+    const uint32_t ch = hash_tokens(wv.ct, key_len, 0x7F4A7C15u);
+    const uint32_t tag = (qgram_tag16(qh) << 16) | (ch >> 16);
     const unsigned long long mine = ((unsigned long long)tag << 32) | (uint32_t)p;
     uint32_t slot = qh & (uint32_t)(slots - 1);
     for (int probe = 0; probe < slots; ++probe) {
@@ -88,16 +119,10 @@ __device__ __forceinline__ bool index_insert(IndexEntry* tbl, int slots, const i
             }
             cur = old;
         }
-        if ((uint32_t)(cur >> 32) == tag) {
-            const int rp = (int)(uint32_t)cur;
-            bool same = true;
-            for (int t = 1; t <= q && same; ++t) same = h[rp - t] == h[p - t];
-            for (int t = 0; t < key_len && same; ++t) same = h[rp + t] == h[p + t];
-            if (same) {
-                atomicAdd(&tbl[slot].count, 1);
-                atomicMax(&tbl[slot].last, p);
-                return true;
-            }
+        if ((uint32_t)(cur >> 32) == tag && same_window(wv, h, (int)(uint32_t)cur, q, key_len)) {
+            atomicAdd(&tbl[slot].count, 1);
+            atomicMax(&tbl[slot].last, p);
+            return true;
         }
         slot = (slot + 1) & (uint32_t)(slots - 1);
     }
@@ -142,7 +167,9 @@ __global__ void index_build_kernel(IndexView ix, const int32_t* __restrict__ his
         }
         const int q = ix.qs[qi];
         if (p < q || p + ix.w > L) continue;
-        if (!index_insert(ix.tables + ((size_t)s * ix.n_q + qi) * ix.slots, ix.slots, hist + (size_t)s * ix.cap, p, q, ix.key_len)) {
+        const int32_t* h = hist + (size_t)s * ix.cap;
+        const Window wv = load_window(h, p, q, ix.key_len);
+        if (!index_insert(ix.tables + ((size_t)s * ix.n_q + qi) * ix.slots, ix.slots, h, wv, p, q, ix.key_len)) {
             ix.state[2 * s + 1] = 0;
             atomicOr(status, SPEC_STATUS_INDEX);
         }
@@ -182,7 +209,8 @@ __global__ void __launch_bounds__(128) accept_commit_index_kernel(const AcceptAr
     for (int item = lane; item < n_new * ix.n_q; item += 32) {
         const int p = p_lo + item / ix.n_q, qi = item % ix.n_q, q = ix.qs[qi];
         if (p < q) continue;
-        ok = index_insert(ix.tables + ((size_t)s * ix.n_q + qi) * ix.slots, ix.slots, h, p, q, ix.key_len) && ok;
+        const Window wv = load_window(h, p, q, ix.key_len);
+        ok = index_insert(ix.tables + ((size_t)s * ix.n_q + qi) * ix.slots, ix.slots, h, wv, p, q, ix.key_len) && ok;
     }
     ok = __all_sync(0xffffffffu, ok);
     if (lane == 0) {
@@ -276,8 +304,11 @@ __global__ void __launch_bounds__(kIndexThreads) draft_index_kernel(const DraftP
             const int q = P.qs[qi];
             if (L < q + P.w) continue;  // no complete window yet
             const IndexEntry* tbl = ix.tables + ((size_t)s * ix.n_q + qmap[qi]) * ix.slots;
-            const uint32_t qh = hash_tokens(h + L - q, q, 0x9E3779B9u);
-            const uint32_t qtag = fmix32(qh + 0x632BE5ABu) >> 16;
+            int qg[kMaxQ];
+#pragma unroll
+            for (int t = 0; t < kMaxQ; ++t) qg[t] = sm->tq[t];  // tq[t] = the token t + 1 places before the end
+            const uint32_t qh = qgram_hash(qg, q);
+            const uint32_t qtag = qgram_tag16(qh);
             const uint32_t home = qh & (uint32_t)(ix.slots - 1);
             for (int it = 0; it * 32 < ix.slots; ++it) {
                 const IndexEntry e = tbl[(home + it * 32 + lane) & (uint32_t)(ix.slots - 1)];
@@ -287,7 +318,11 @@ __global__ void __launch_bounds__(kIndexThreads) draft_index_kernel(const DraftP
                 bool match = before_end && !empty && (uint32_t)(e.key >> 48) == qtag;
                 if (match) {
                     const int rp = (int)(uint32_t)e.key;
-                    for (int t = 1; t <= q && match; ++t) match = h[rp - t] == h[L - t];
+                    int diff = 0;
+#pragma unroll
+                    for (int t = 0; t < kMaxQ; ++t)
+                        if (t < q) diff |= h[rp - 1 - t] ^ qg[t];
+                    match = diff == 0;
                 }
                 if (match) {
                     const int idx = atomicAdd(&sm->n_keys, 1);
