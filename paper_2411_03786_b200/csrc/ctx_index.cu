@@ -181,41 +181,94 @@ __global__ void index_mark_valid_kernel(IndexView ix) {
     if (s < ix.S) ix.state[2 * s + 1] = 1;
 }
 
+// The same insertion by a whole warp (every lane holds the same window): the probe run is read 32 slots at a
+// time, so a q-gram with hundreds of groups costs a few steps, not hundreds of dependent loads.  Safe against
+// other warps inserting into the same table.
+__device__ __forceinline__ bool index_insert_warp(IndexEntry* tbl, int slots, const int32_t* h, const Window& wv, int p, int q, int key_len,
+                                                  int lane) {
+    const uint32_t qh = qgram_hash(wv.qg, q);
+    const uint32_t ch = hash_tokens(wv.ct, key_len, 0x7F4A7C15u);
+    const uint32_t tag = (qgram_tag16(qh) << 16) | (ch >> 16);
+    const unsigned long long mine = ((unsigned long long)tag << 32) | (uint32_t)p;
+    const uint32_t home = qh & (uint32_t)(slots - 1);
+    int retries = 0;
+    for (int it = 0; it * 32 < slots; ++it) {
+        const uint32_t slot = (home + it * 32 + lane) & (uint32_t)(slots - 1);
+        const unsigned long long cur = *((volatile unsigned long long*)&tbl[slot].key);
+        const bool empty = cur == kIndexEmpty;
+        const unsigned eb = __ballot_sync(0xffffffffu, empty);
+        const bool before_end = eb == 0u || lane < __ffs(eb) - 1;  // the run ends at its first empty slot
+        const bool found = before_end && (uint32_t)(cur >> 32) == tag && same_window(wv, h, (int)(uint32_t)cur, q, key_len);
+        const unsigned fb = __ballot_sync(0xffffffffu, found);
+        if (fb) {
+            if (lane == __ffs(fb) - 1) {
+                atomicAdd(&tbl[slot].count, 1);
+                atomicMax(&tbl[slot].last, p);
+            }
+            return true;
+        }
+        if (eb) {  // the group is new: it takes the slot that ends the run
+            const int first = __ffs(eb) - 1;
+            unsigned long long old = 0ull;
+            if (lane == first) old = atomicCAS(&tbl[slot].key, kIndexEmpty, mine);
+            old = __shfl_sync(0xffffffffu, old, first);
+            if (old == kIndexEmpty) {
+                if (lane == first) {
+                    atomicAdd(&tbl[slot].count, 1);
+                    atomicMax(&tbl[slot].last, p);
+                }
+                return true;
+            }
+            if (++retries > 64) return false;
+            --it;  // another warp took that slot meanwhile: look at these 32 slots again
+        }
+    }
+    return false;
+}
+
 // Greedy acceptance and commit (as accept_commit_kernel), then the windows that the committed tokens completed
-// are added to the index: one warp per sequence, one (window, query length) pair per lane at a time.
+// are added to the index.  One CTA of four warps per sequence: warp 0 accepts and commits, then every warp
+// inserts some of the (window, query length) pairs, a pair at a time.
 __global__ void __launch_bounds__(128) accept_commit_index_kernel(const AcceptArgs a, IndexView ix) {
-    const int lane = threadIdx.x & 31;
-    const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    __shared__ int sh_old, sh_new, sh_fail;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int s = blockIdx.x;
     grid_launch_dependents();
     grid_dependency_wait();
-    if (s >= a.S) return;
-    const int L_old = a.len[s];
-    __syncwarp();
-    accept_sequence(a, s, lane);
-    __threadfence();
-    __syncwarp();  // the committed tokens and the new length are visible to the whole warp
-    const int L_new = *((volatile int*)&a.len[s]);
+    if (warp == 0) {
+        const int L_old = a.len[s];
+        __syncwarp();
+        accept_sequence(a, s, lane);
+        __threadfence();
+        __syncwarp();  // the committed tokens and the new length are visible to the whole warp
+        if (lane == 0) {
+            sh_old = L_old;
+            sh_new = *((volatile int*)&a.len[s]);
+            sh_fail = 0;
+        }
+    }
+    __syncthreads();  // ... and, through the fence above, to the whole CTA
+    const int L_old = sh_old, L_new = sh_new;
     int* st = ix.state + 2 * s;
     const bool in_step = st[1] != 0 && st[0] == L_old && L_old >= 0 && L_new <= ix.cap;
-    __syncwarp();
+    __syncthreads();
     if (!in_step) {  // not built, or the history moved without the index: it stays unusable until it is rebuilt
-        if (lane == 0) st[1] = 0;
+        if (threadIdx.x == 0) st[1] = 0;
         return;
     }
     if (L_new == L_old) return;  // nothing was committed (no room)
-    const int32_t* h = a.hist + (size_t)s * a.cap;  // (written by this warp a moment ago: plain loads)
+    const int32_t* h = a.hist + (size_t)s * a.cap;  // (written a moment ago: plain loads)
     const int p_lo = L_old - ix.w + 1, n_new = L_new - L_old;  // continuation starts p_lo .. p_lo + n_new - 1
-    bool ok = true;
-    for (int item = lane; item < n_new * ix.n_q; item += 32) {
+    for (int item = warp; item < n_new * ix.n_q; item += 4) {
         const int p = p_lo + item / ix.n_q, qi = item % ix.n_q, q = ix.qs[qi];
         if (p < q) continue;
         const Window wv = load_window(h, p, q, ix.key_len);
-        ok = index_insert(ix.tables + ((size_t)s * ix.n_q + qi) * ix.slots, ix.slots, h, wv, p, q, ix.key_len) && ok;
+        if (!index_insert_warp(ix.tables + ((size_t)s * ix.n_q + qi) * ix.slots, ix.slots, h, wv, p, q, ix.key_len, lane) && lane == 0) sh_fail = 1;
     }
-    ok = __all_sync(0xffffffffu, ok);
-    if (lane == 0) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
         st[0] = L_new;
-        if (!ok) {
+        if (sh_fail) {
             st[1] = 0;
             atomicOr(a.status, SPEC_STATUS_INDEX);
         }
@@ -426,8 +479,7 @@ int launch_index_build(spec_ctx* ctx, void* d_index, const int32_t* d_hist, cons
 
 int launch_accept_indexed(spec_ctx* ctx, const AcceptArgs& a, cudaStream_t st) {
     const IndexView ix = make_view(ctx->index);
-    const int warps = 4;
-    cudaError_t e = launch_pdl(accept_commit_index_kernel, dim3((a.S + warps - 1) / warps), dim3(warps * 32), 0, st, a, ix);
+    cudaError_t e = launch_pdl(accept_commit_index_kernel, dim3((unsigned)a.S), dim3(128), 0, st, a, ix);
     ctx->launches += 1;
     return check_cuda(ctx, e, "accept_and_commit_indexed launch");
 }
