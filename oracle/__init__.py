@@ -23,6 +23,7 @@ _lib = None
 FLAG_DEDUP = 1
 FLAG_MODEL_FILL = 2
 FLAG_KEY_NEXT_TOKEN = 4
+FLAG_PARTIAL_TAIL = 8
 
 
 def flag_reserve(n: int) -> int:
@@ -85,6 +86,19 @@ def context_draft(hist, q: int, w: int, topk: int, key_len: int | None = None):
     n = lib().oracle_context_draft_keyed(_p(hist, C.c_int32), int(hist.size), int(q), int(w),
                                          int(w if key_len is None else key_len), int(topk),
                                          _p(rows, C.c_int32), _p(counts, C.c_int32), _p(lasts, C.c_int32))
+    return rows[:n].copy(), counts[:n].copy(), lasts[:n].copy()
+
+
+def context_draft_partial(hist, q: int, w: int, topk: int, key_len: int | None = None):
+    """The variant in which occurrences with fewer than w following tokens count too, their continuation
+    extended periodically.  Returns ``(rows[n, w], counts[n], last_start[n])`` with n <= topk."""
+    hist = _i32(hist)
+    rows = np.full((max(topk, 1), w), -1, dtype=np.int32)
+    counts = np.zeros(max(topk, 1), dtype=np.int32)
+    lasts = np.zeros(max(topk, 1), dtype=np.int32)
+    n = lib().oracle_context_draft_partial(_p(hist, C.c_int32), int(hist.size), int(q), int(w),
+                                           int(w if key_len is None else key_len), int(topk),
+                                           _p(rows, C.c_int32), _p(counts, C.c_int32), _p(lasts, C.c_int32))
     return rows[:n].copy(), counts[:n].copy(), lasts[:n].copy()
 
 

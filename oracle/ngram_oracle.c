@@ -127,6 +127,66 @@ int oracle_context_draft_keyed(const int32_t* hist, int L, int q, int w, int key
     return n_out;
 }
 
+/* A variant the paper does not have (its listing slides full windows only, which hides the most recent
+ * repeats): occurrences of the query with fewer than w tokens after them count too.  Such an occurrence at
+ * window start i has d = L - (i + q) >= 1 following tokens; its continuation is read as if the history went
+ * on repeating them: c[t] = hist[i + q + (t mod d)] once i + q + t reaches L (the way an overlapping copy
+ * extends itself).  For a window with w tokens after it this is the plain continuation.  Grouping, counts,
+ * `last` and the order are as in oracle_context_draft_keyed, over the windows i = 0 .. L - q - 1. */
+static int32_t wrapped_token(const int32_t* hist, int L, int p, int t) {
+    return p + t < L ? hist[p + t] : hist[p + t % (L - p)];
+}
+
+int oracle_context_draft_partial(const int32_t* hist, int L, int q, int w, int key_len, int topk,
+                                 int32_t* rows, int32_t* counts, int32_t* lasts) {
+    if (q < 1 || w < 1 || topk < 1 || L < q + 1) return 0;
+    const int32_t* query = hist + (L - q);
+    int n_windows = L - q; /* i = 0 .. L - q - 1: at least one token follows, and the query itself is not a window */
+    int* g_first = (int*)malloc(sizeof(int) * (size_t)n_windows);
+    int* g_count = (int*)malloc(sizeof(int) * (size_t)n_windows);
+    int* g_last = (int*)malloc(sizeof(int) * (size_t)n_windows);
+    char* g_taken = (char*)calloc((size_t)n_windows, 1);
+    int n_groups = 0;
+    for (int i = 0; i < n_windows; ++i) {
+        int match = 1;
+        for (int t = 0; t < q; ++t)
+            if (hist[i + t] != query[t]) { match = 0; break; }
+        if (!match) continue;
+        int g = -1;
+        for (int j = 0; j < n_groups && g < 0; ++j) {
+            int same = 1;
+            for (int t = 0; t < key_len; ++t)
+                if (wrapped_token(hist, L, i + q, t) != wrapped_token(hist, L, g_first[j] + q, t)) { same = 0; break; }
+            if (same) g = j;
+        }
+        if (g < 0) {
+            g = n_groups++;
+            g_first[g] = i;
+            g_count[g] = 0;
+            g_last[g] = i;
+        }
+        g_count[g] += 1;
+        if (i > g_last[g]) g_last[g] = i;
+    }
+    int n_out = 0;
+    while (n_out < topk && n_out < n_groups) {
+        int best = -1;
+        for (int j = 0; j < n_groups; ++j) {
+            if (g_taken[j]) continue;
+            if (best < 0 || g_count[j] > g_count[best] ||
+                (g_count[j] == g_count[best] && g_last[j] > g_last[best]))
+                best = j;
+        }
+        g_taken[best] = 1;
+        for (int t = 0; t < w; ++t) rows[n_out * w + t] = wrapped_token(hist, L, g_last[best] + q, t);
+        if (counts) counts[n_out] = g_count[best];
+        if (lasts) lasts[n_out] = g_last[best];
+        ++n_out;
+    }
+    free(g_first); free(g_count); free(g_last); free(g_taken);
+    return n_out;
+}
+
 /* ------------------------------------------------------------------ extended model bigram (Section 4.1, "Extensions")
  *
  * T[V, k_tab] holds, per token x, the k_tab most likely next tokens of the model
@@ -151,7 +211,8 @@ void oracle_extend_table(const int32_t* T, int V, int k_tab, int w, int32_t* ext
  * in the caller's priority order, at most topk rows each; then, if asked, the
  * extended model bigram of the last token in rank order.  With dedup a row equal
  * in all w tokens to one already taken is skipped.  Unused rows are -1.
- * flags: bit0 = dedup, bit1 = model fill, bit2 = group matches by their next token only, bits 8..15 = rows reserved for the model strategy (the
+ * flags: bit0 = dedup, bit1 = model fill, bit2 = group matches by their next token only, bit3 = occurrences with fewer than w
+ * following tokens count too (oracle_context_draft_partial), bits 8..15 = rows reserved for the model strategy (the
  * context strategies together take at most B minus that many rows; the paper leaves the
  * allocation between strategies open, Section 5.2).
  * src[b] = q of the strategy that produced row b, 0 for the model, -1 unused.
@@ -168,7 +229,8 @@ int oracle_draft_sequence(const int32_t* hist, int L, const int* qs, int n_q, in
     int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > k_tab ? topk : k_tab) * (size_t)w);
     int32_t* cnt = (int32_t*)malloc(sizeof(int32_t) * (size_t)(topk > 0 ? topk : 1));
     for (int qi = 0; qi < n_q && n < ctx_cap; ++qi) {
-        int m = oracle_context_draft_keyed(hist, L, qs[qi], w, (flags & 4) ? 1 : w, topk, cand, cnt, NULL);
+        int m = (flags & 8) ? oracle_context_draft_partial(hist, L, qs[qi], w, (flags & 4) ? 1 : w, topk, cand, cnt, NULL)
+                            : oracle_context_draft_keyed(hist, L, qs[qi], w, (flags & 4) ? 1 : w, topk, cand, cnt, NULL);
         for (int r = 0; r < m && n < ctx_cap; ++r) {
             int dup = 0;
             /* The paper's tokens are elements of the vocabulary by definition (Section 2).  When the

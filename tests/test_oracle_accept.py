@@ -115,11 +115,15 @@ def brute_context_next_token(hist, q, w, topk):
 
 
 def brute_mix(hist, qs, topk, B, w, flags, T):
-    from test_oracle_context import brute_context
+    from test_oracle_context import brute_context, brute_context_partial
     rows, src, cnt = [], [], []
     ctx_cap = max(0, B - ((flags >> 8) & 0xFF))
     for q in qs:
-        for c, n, _ in (brute_context(hist, q, w, topk) if not flags & 4 else brute_context_next_token(hist, q, w, topk)):
+        if flags & 8:       # occurrences near the end count too
+            found = brute_context_partial(hist, q, w, topk, 1 if flags & 4 else w)
+        else:
+            found = brute_context(hist, q, w, topk) if not flags & 4 else brute_context_next_token(hist, q, w, topk)
+        for c, n, _ in found:
             if len(rows) >= ctx_cap:
                 break
             if (flags & 1) and list(c) in rows:
@@ -150,7 +154,7 @@ def test_mixing_against_brute_force():
         n_q = int(g.integers(0, 4))
         qs = [int(q) for q in g.permutation([1, 2, 3, 4])[:n_q]]
         topk, B, w = int(g.integers(1, 5)), int(g.integers(1, 9)), int(g.integers(1, 5))
-        flags = int(g.integers(0, 8)) | (oracle.flag_reserve(int(g.integers(0, B + 2))) if trial % 3 == 0 else 0)
+        flags = int(g.integers(0, 16)) | (oracle.flag_reserve(int(g.integers(0, B + 2))) if trial % 3 == 0 else 0)
         cap = (L + 3) // 4 * 4 + 4
         h2 = np.full((1, cap), -1, np.int32)
         h2[0, :L] = hist

@@ -144,3 +144,73 @@ def test_next_token_keyed_variant():
     a = oracle.context_draft(hist, 1, 1, 8)
     b = oracle.context_draft(hist, 1, 1, 8, key_len=1)
     assert all(np.array_equal(x, y) for x, y in zip(a, b))
+
+
+# ----------------------------------------------------------------------------- partial continuations near the tail
+def brute_context_partial(hist, q, w, topk, key_len=None):
+    """Dictionary restatement: every occurrence of the last q tokens that has at least one token after it; a
+    continuation that runs past the end of the history repeats the tokens it has."""
+    hist = [int(t) for t in hist]
+    L = len(hist)
+    key_len = w if key_len is None else key_len
+    if L < q + 1:
+        return []
+    groups = {}
+    for i in range(L - q):
+        if hist[i:i + q] != hist[L - q:]:
+            continue
+        p = i + q
+        have = hist[p:]
+        cont = tuple(have[t] if t < len(have) else have[t % len(have)] for t in range(w))
+        cnt, _, _ = groups.get(cont[:key_len], (0, -1, None))
+        groups[cont[:key_len]] = (cnt + 1, i, cont)          # i increases: the latest occurrence supplies the row
+    order = sorted(groups.values(), key=lambda v: (-v[0], -v[1]))[:topk]
+    return [(cont, cnt, last) for cnt, last, cont in order]
+
+
+def test_partial_tail_hand_example():
+    # "1 2 3" repeats; the query is the final "1 2".  Full windows of 2 + 4 tokens: only the one at 0, continuation
+    # 3 1 2 3.  The occurrence at 3 has three tokens after it (3 1 2); continued periodically it reads 3 1 2 3 as
+    # well, so with partial continuations the same row is seen twice, the later time at window start 3.
+    hist = np.array([1, 2, 3, 1, 2, 3, 1, 2], np.int32)
+    rows, counts, lasts = oracle.context_draft(hist, 2, 4, 4)
+    assert rows.tolist() == [[3, 1, 2, 3]] and counts.tolist() == [1] and lasts.tolist() == [0]
+    rows, counts, lasts = oracle.context_draft_partial(hist, 2, 4, 4)
+    assert rows.tolist() == [[3, 1, 2, 3]] and counts.tolist() == [2] and lasts.tolist() == [3]
+    # one token after the occurrence: it alone is repeated
+    hist = np.array([5, 7, 9, 4, 5, 7], np.int32)            # query "7"; occurrence at 1 is followed by 9 4 5 7 ...
+    rows, counts, lasts = oracle.context_draft_partial(hist, 1, 6, 3)
+    assert rows.tolist() == [[9, 4, 5, 7, 9, 4]] and counts.tolist() == [1]
+    hist = np.array([8, 8, 8], np.int32)                      # query "8": occurrences at 0 (followed by 8 8) and 1 (by 8)
+    rows, counts, lasts = oracle.context_draft_partial(hist, 1, 5, 3)
+    assert rows.tolist() == [[8, 8, 8, 8, 8]] and counts.tolist() == [2] and lasts.tolist() == [1]
+
+
+def test_partial_tail_against_brute_force():
+    g = np.random.default_rng(21)
+    for trial in range(900):
+        A = int(g.integers(1, 4))
+        L = int(g.integers(0, 40))
+        hist = g.integers(0, A, L).astype(np.int32)
+        if trial % 3 == 0 and L > 6:                          # periodic tails, where the extension matters most
+            per = int(g.integers(1, 5))
+            hist[L // 2:] = np.resize(hist[L // 2:L // 2 + per], L - L // 2)
+        q, w, topk = int(g.integers(1, 5)), int(g.integers(1, 8)), int(g.integers(1, 6))
+        key_len = 1 if trial % 4 == 0 else w
+        want = brute_context_partial(hist, q, w, topk, key_len)
+        rows, counts, lasts = oracle.context_draft_partial(hist, q, w, topk, key_len)
+        assert rows.tolist() == [list(c) for c, _, _ in want]
+        assert counts.tolist() == [n for _, n, _ in want] and lasts.tolist() == [i for _, _, i in want]
+
+
+def test_partial_tail_reduces_to_the_plain_rule_when_no_occurrence_is_near_the_end():
+    g = np.random.default_rng(22)
+    for _ in range(200):
+        L, q, w = int(g.integers(20, 60)), int(g.integers(1, 4)), int(g.integers(1, 7))
+        hist = g.integers(0, 3, L).astype(np.int32)
+        hist[L - q:] = 9                                       # the query occurs nowhere else ...
+        pos = int(g.integers(0, L - q - w - q + 1)) if L - q - w - q + 1 > 0 else 0
+        hist[pos:pos + q] = 9                                  # ... except once, far enough from the end
+        a = oracle.context_draft(hist, q, w, 5)
+        b = oracle.context_draft_partial(hist, q, w, 5)
+        assert all(np.array_equal(x, y) for x, y in zip(a, b))
