@@ -67,7 +67,7 @@ enum {
 };
 
 enum { SPEC_F32 = 0, SPEC_BF16 = 1 };
-enum { SPEC_FLAG_DEDUP = 1, SPEC_FLAG_MODEL_FILL = 2, SPEC_FLAG_KEY_NEXT_TOKEN = 4 };
+enum { SPEC_FLAG_DEDUP = 1, SPEC_FLAG_MODEL_FILL = 2, SPEC_FLAG_KEY_NEXT_TOKEN = 4, SPEC_FLAG_PARTIAL_TAIL = 8 };
 /* OR into the draft flags to reserve n (0..255) of the B draft rows for the model strategy */
 #define SPEC_FLAG_RESERVE(n) (((n) & 0xFF) << 8)
 enum { SPEC_MAX_VERIFY_ROWS = 65536 };
@@ -150,6 +150,10 @@ int spec_set_model_table(spec_ctx* ctx, const int32_t* d_tab_idx, int k_tab, con
  * an open knob in the paper, Section 5.2); a model row is then compared with the rows taken only.
  * SPEC_FLAG_KEY_NEXT_TOKEN groups the matches by their next token only (counting "the tokens that
  * follow each occurrence"); the row of a group is then the w tokens after its latest occurrence.
+ * SPEC_FLAG_PARTIAL_TAIL also counts the occurrences that have fewer than w (but at least one) tokens
+ * after them - the most recent repeats, which full windows cannot see; such a continuation is read as if
+ * the history went on repeating the tokens it has (token t beyond the end = token t mod d of the d that
+ * exist).  Histories then need q + 1 tokens to give rows for q.  Not available from the context index.
  *   qs         host array of n_q query lengths (n_q = 0: model rows only).
  *   d_drafts   [S, B, w] out, unused rows = -1.      d_ndrafts [S] out.
  *   d_src      [S, B] out or NULL: q of the producing strategy, 0 = model, -1 = unused.

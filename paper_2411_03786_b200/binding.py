@@ -9,7 +9,7 @@ import torch
 
 from .build import LIB, build_library
 
-FLAG_DEDUP, FLAG_MODEL_FILL, FLAG_KEY_NEXT_TOKEN = 1, 2, 4
+FLAG_DEDUP, FLAG_MODEL_FILL, FLAG_KEY_NEXT_TOKEN, FLAG_PARTIAL_TAIL = 1, 2, 4, 8
 STATUS_TOKEN_RANGE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_GROUPS, STATUS_INDEX = 1, 2, 4, 8, 16
 SPEC_F32, SPEC_BF16 = 0, 1
 

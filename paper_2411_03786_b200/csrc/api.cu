@@ -307,6 +307,8 @@ int draft_context_ngrams_indexed(spec_ctx* ctx, const void* d_index, const int32
     if (!d_index || d_index != m.ptr) return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: d_index is not the index registered by spec_context_index_build");
     if (S != m.S || cap != m.cap || w != m.w || ((flags & SPEC_FLAG_KEY_NEXT_TOKEN) ? 1 : w) != m.key_len)
         return fail(ctx, SPEC_ERR_ARG, "draft_context_ngrams_indexed: S, cap, w and the key flag must be those the index was built with");
+    if (flags & SPEC_FLAG_PARTIAL_TAIL)
+        return fail(ctx, SPEC_ERR_UNSUPPORTED, "draft_context_ngrams_indexed: the index holds complete windows only (SPEC_FLAG_PARTIAL_TAIL needs draft_context_ngrams)");
     if ((flags & SPEC_FLAG_MODEL_FILL) && !ctx->tab_idx)
         return fail(ctx, SPEC_ERR_NOT_BUILT, "draft_context_ngrams_indexed: model fill needs build_model_ngram_tables first");
     cudaSetDevice(ctx->device);

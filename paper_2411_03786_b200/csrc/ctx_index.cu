@@ -444,9 +444,9 @@ __global__ void __launch_bounds__(kIndexThreads) draft_index_kernel(const DraftP
                 break;
             }
         }
-        mix_and_emit(P, s, h, gave_up, X, tid, NT, sync);
+        mix_and_emit(P, s, h, L, gave_up, X, tid, NT, sync);
     } else {
-        mix_and_emit(P, s, h, false, X, tid, NT, sync);
+        mix_and_emit(P, s, h, L, false, X, tid, NT, sync);
     }
 }
 

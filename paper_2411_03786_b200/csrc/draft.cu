@@ -533,12 +533,16 @@ int launch_draft(spec_ctx* ctx, const int32_t* d_hist, const int32_t* d_len, int
     // cannot fill the GPU (with many sequences the team kernel streams them)
     unsigned csize = 1;
     while (csize < 8 && (int)(csize * 2) * 16384 <= cap && (long long)S * (csize * 2) <= ctx->num_sms) csize <<= 1;
-    const bool stage = csize == 1 && cap <= 8192;
+    // (continuations that run past the end of the history are the batch kernels' business: this kernel carries
+    // only the paper's rule)
+    const bool partial = (flags & SPEC_FLAG_PARTIAL_TAIL) != 0;
+    if (partial) csize = 1;
+    const bool stage = csize == 1 && cap <= 8192 && !partial;
     if (csize == 1) {
         // Batches: histories of up to 16384 tokens are staged in shared memory by warp teams (when the batch
         // fills the GPU more than twice over, or a history is too long for the staging of this kernel);
         // longer ones are streamed by the scanner / finisher kernel.
-        const bool batch = S > 2 * ctx->num_sms;
+        const bool batch = S > 2 * ctx->num_sms || partial;
         if (cap <= 16384 && (batch || !stage)) {
             const int rc = launch_draft_team(ctx, P, st);
             if (rc != kDraftNoFit) return rc;  // (the largest draft shapes leave no room for the staged history)

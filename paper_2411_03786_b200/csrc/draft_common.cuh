@@ -53,13 +53,21 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
     return v;
 }
 
+// Token t of the continuation that starts at p.  With SPEC_FLAG_PARTIAL_TAIL (Lw = history length, else 0) a
+// continuation that runs past the end of the history repeats the tokens it has.
+__device__ __forceinline__ int cont_tok(const int32_t* __restrict__ h, int Lw, int p, int t) {
+    int i = p + t;
+    if (Lw != 0 && i >= Lw) i = p + t % (Lw - p);
+    return h[i];
+}
+
 // Group the match whose continuation starts at p (query index qi) in an open-addressing table:
 // rep[slot] = (qi << 28 | start of the group's first-seen continuation), cnt, last; a collision is
 // resolved by comparing the actual tokens, so grouping is exact.  n_groups / overflow are the table's
 // counters; once overflow is set the pass is void and nothing more is inserted.
 __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int p, int qi, int key_len, uint32_t hsh,
                                              int slots, int max_groups, int* rep, int* cnt, int* last,
-                                             int* grp_slot, int* n_groups, int* overflow) {
+                                             int* grp_slot, int* n_groups, int* overflow, int Lw = 0) {
     if (*((volatile int*)overflow)) return;  // this pass is void already: do not fill the table further
     uint32_t slot = hsh & (uint32_t)(slots - 1);
     const int me = (qi << 28) | p;
@@ -84,7 +92,7 @@ __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int 
             const int rp = cur & 0x0FFFFFFF;
             bool same = true;
             for (int t = 0; t < key_len; ++t)
-                if (h[rp + t] != h[p + t]) {
+                if (cont_tok(h, Lw, rp, t) != cont_tok(h, Lw, p, t)) {
                     same = false;
                     break;
                 }
@@ -159,6 +167,8 @@ __device__ __forceinline__ int scan_pass(const DraftParams& P, const int32_t* __
     const int n_scan = L - w;  // token index x = p - 1 runs over [0, n_scan)
     const int key_len = (P.flags & SPEC_FLAG_KEY_NEXT_TOKEN) ? 1 : w;
     const bool need2 = P.q_min >= 2;  // every query has at least two tokens: test the second one in registers
+    const bool partial = (P.flags & SPEC_FLAG_PARTIAL_TAIL) != 0;  // occurrences with fewer than w following tokens count too
+    const int Lw = partial ? L : 0;
     const int4* h4 = reinterpret_cast<const int4*>(h);
     const int n_vec = (max(n_scan, 0) + 3) >> 2;
     // bits of one vector; `before` is the token left of the vector's first one
@@ -186,13 +196,13 @@ __device__ __forceinline__ int scan_pass(const DraftParams& P, const int32_t* __
         }
         const int p = x + 1;
         uint32_t hc = 0x9E3779B9u;  // one multiply-add per token, mixed once per query length below
-        for (int t = 0; t < key_len; ++t) hc = hc * 0x85EBCA6Bu + (uint32_t)h[p + t];
+        for (int t = 0; t < key_len; ++t) hc = hc * 0x85EBCA6Bu + (uint32_t)cont_tok(h, Lw, p, t);
         for (int qi = 0; qi < P.n_q; ++qi) {
             const int q = P.qs[qi];
-            if (m < q || L < q + w) continue;
+            if (m < q || (!partial && L < q + w)) continue;
             const uint32_t hq = fmix32(hc + (uint32_t)qi * 0x632BE5ABu);
             if (R > 1 && (int)(fmix32(hq ^ 0xA511E9B3u) % (uint32_t)R) != r) continue;
-            insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, T.rep, T.cnt, T.last, T.grp_slot, T.n_groups, T.overflow);
+            insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, T.rep, T.cnt, T.last, T.grp_slot, T.n_groups, T.overflow, Lw);
         }
     };
     int qn = 0;  // queued matches (the same in every lane)
@@ -290,6 +300,10 @@ __device__ __forceinline__ int scan_pass(const DraftParams& P, const int32_t* __
     if (need2) scan_blocks(std::true_type{});
     else scan_blocks(std::false_type{});
     flush_matches();
+    if (partial && tid < 32) {  // the last w - 1 positions, by the group's first warp: continuations that run past the end
+        for (int x = max(n_scan, 0) + lane; x <= L - 2; x += 32)
+            if (h[x] == t0) handle_match(x);
+    }
     return reached;
 }
 
@@ -447,9 +461,10 @@ __device__ __forceinline__ void rank_pass(const DraftParams& P, const DraftTable
 // Mixed allocation of sequence s: context rows in query order, then model rows by rank; duplicates dropped;
 // the first B survivors become the drafts.  Writes the four outputs.  Starts and ends with a barrier.
 template <class Sync>
-__device__ __forceinline__ void mix_and_emit(const DraftParams& P, int s, const int32_t* __restrict__ h, bool gave_up,
+__device__ __forceinline__ void mix_and_emit(const DraftParams& P, int s, const int32_t* __restrict__ h, int L, bool gave_up,
                                              const DraftScratch& X, int tid, int nthr, Sync&& sync) {
     const int w = P.w, topk = P.topk, lane = tid & 31, warp = tid >> 5;
+    const int Lw = (P.flags & SPEC_FLAG_PARTIAL_TAIL) ? L : 0;
     const bool dedup = (P.flags & SPEC_FLAG_DEDUP) != 0;
     sync();
     if (tid == 0) {
@@ -481,13 +496,13 @@ __device__ __forceinline__ void mix_and_emit(const DraftParams& P, int s, const 
         } else {
             const unsigned long long key = X.run_key[li * topk + r];
             const int start = (int)(uint32_t)key;
-            tok = h[start + t];
+            tok = cont_tok(h, Lw, start, t);
             src = P.qs[li];
             count = (int)(key >> 32);
             if (t == 0) {  // a context row that carries a token outside the vocabulary is dropped
                 bool in_range = true;
                 for (int u = 0; u < w; ++u) {
-                    const int tk = h[start + u];
+                    const int tk = cont_tok(h, Lw, start, u);
                     in_range = in_range && tk >= 0 && tk < P.V;
                 }
                 keep = in_range ? 1 : 0;

@@ -111,9 +111,10 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) draft_stream_kernel(const D
             named_arrive(BAR_FEMPTY + k, FETCH_COUNT);
             k ^= 1;
             const int32_t* __restrict__ h = P.hist + (size_t)s * P.cap;
+            const bool partial = (P.flags & SPEC_FLAG_PARTIAL_TAIL) != 0;
             bool any_q = false;
-            for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + P.w);
-            const bool scan = any_q && L - P.w >= 1;
+            for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + (partial ? 1 : P.w));
+            const bool scan = any_q && (L - P.w >= 1 || (partial && L >= 2));
             int R = 1;
             for (;;) {
                 bool overflowed = false;
@@ -199,7 +200,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) draft_stream_kernel(const D
             if (!(flags & PASS_VOID)) rank_pass(P, table(buf), X, tid, PWT, post_sync);
             else post_sync();
             release(buf);  // the winners live in run_key: the scanners may fill this table again
-            if ((flags & PASS_LAST) && !(flags & PASS_VOID)) mix_and_emit(P, s, h, (flags & PASS_GAVE_UP) != 0, X, tid, PWT, post_sync);
+            if ((flags & PASS_LAST) && !(flags & PASS_VOID)) mix_and_emit(P, s, h, L, (flags & PASS_GAVE_UP) != 0, X, tid, PWT, post_sync);
             buf ^= 1;
         }
     } else {

@@ -149,11 +149,12 @@ __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(cons
         // ---- context N-grams
         const int n_scan = L - P.w;
         const int t0 = sm->tq[0], t1 = sm->tq[1], t2 = sm->tq[2], t3 = sm->tq[3];
+        const bool partial = (P.flags & SPEC_FLAG_PARTIAL_TAIL) != 0;
         bool any_q = false;
-        for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + P.w);
+        for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + (partial ? 1 : P.w));
         int R = 1;
         bool gave_up = false;
-        while (any_q && n_scan >= 1) {
+        while (any_q && (n_scan >= 1 || (partial && L >= 2))) {
             team_sync();
             if (tid < kMaxNQ) sm->n_run[tid] = 0;
             bool overflowed = false;
@@ -184,7 +185,7 @@ __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(cons
                 break;
             }
         }
-        mix_and_emit(P, s, h, gave_up, X, tid, TT, team_sync);
+        mix_and_emit(P, s, h, L, gave_up, X, tid, TT, team_sync);
     }
 
     // The CTA that leaves last re-arms the work counter for the next batch.  (Every CTA has stopped taking

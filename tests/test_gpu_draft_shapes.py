@@ -46,6 +46,11 @@ def test_random_draft_problem(ctx, case):
     topk = int(g.integers(1, B + 1))
     k_tab = int(g.integers(1, 17))
     flags = int(g.choice([0, 1, 2, 3, 7, 5])) | (ngs.flag_reserve(int(g.integers(0, B + 1))) if g.random() < 0.3 else 0)
+    if case % 4 == 3:
+        flags |= ngs.FLAG_PARTIAL_TAIL          # occurrences near the end count too (served by the batch kernels)
+        if lens[0] > 30:                        # ... and a periodic tail makes them matter
+            per = int(g.integers(1, 7))
+            hist[0, lens[0] - 25:lens[0]] = np.resize(hist[0, lens[0] - 25:lens[0] - 25 + per], 25)
     T = np.stack([g.permutation(V)[:k_tab] for _ in range(V)]).astype(np.int32)
     ext = oracle.extend_table(T, w) if g.random() < 0.5 else None
     ctx.set_model_table(dev_i32(T), dev_i32(ext) if ext is not None else None)
@@ -123,4 +128,35 @@ def test_batches_across_team_sizes(ctx, S, Lmax, alpha, qs, flags):
         got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, fl)
         for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
             assert np.array_equal(a.cpu().numpy(), b), name
+    assert ctx.get_status() == 0
+
+
+@pytest.mark.parametrize("S,Lmax,qs,w,flags", [(5, 60, [1, 2], 6, 11), (40, 900, [3, 2, 1], 9, 15), (700, 300, [2], 5, 9),
+                                               (3, 12000, [1, 3], 8, 11), (200, 20000, [2, 1], 7, 11), (2, 70000, [4, 2], 16, 9)])
+def test_occurrences_with_partial_continuations(ctx, S, Lmax, qs, w, flags):
+    """SPEC_FLAG_PARTIAL_TAIL on histories that end in a repeating pattern (period 1 to 2 w): the occurrences that
+    decide the draft are the ones closer than w to the end.  Staged teams, scanner / finisher warps, single sequences
+    and batches; lengths down to below a window."""
+    g = np.random.default_rng(77000 + S + Lmax)
+    B, topk, k_tab = 12, 6, 5
+    cap = (Lmax + 11) // 4 * 4
+    lens = np.array([Lmax if s % 3 == 0 else int(g.integers(0, Lmax + 1)) for s in range(S)], np.int32)
+    lens[-1] = min(Lmax, int(g.integers(1, w + 2)))            # shorter than a window
+    hist = np.full((S, cap), -1, np.int32)
+    n_diff = 0
+    for s in range(S):
+        h = g.integers(0, 6, lens[s])
+        per = int(g.integers(1, 2 * w + 1))
+        tail = min(int(lens[s]), per * int(g.integers(2, 6)))
+        if tail > per:
+            h[lens[s] - tail:] = np.resize(h[lens[s] - tail:lens[s] - tail + per], tail)
+        hist[s, :lens[s]] = h
+    T = np.stack([g.permutation(V)[:k_tab] for _ in range(V)]).astype(np.int32)
+    ctx.set_model_table(dev_i32(T), None)
+    want = oracle.draft_batch(hist, lens, qs, topk, B, w, flags, T)
+    plain = oracle.draft_batch(hist, lens, qs, topk, B, w, flags & ~8, T)
+    assert not np.array_equal(want[0], plain[0])                 # the flag changes the drafts on these histories
+    got = ctx.draft_context_ngrams(dev_i32(hist), dev_i32(lens), qs, topk, B, w, flags)
+    for a, b, name in zip(got, want, ("drafts", "n_drafts", "src", "counts")):
+        assert np.array_equal(a.cpu().numpy(), b), name
     assert ctx.get_status() == 0
