@@ -784,6 +784,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the sweep of verify block heights across the tile steps")
     ap.add_argument("--no-fp8", action="store_true", help="skip timing the 8-bit (E4M3) verification head (reported beside the bf16 numbers)")
     ap.add_argument("--no-graph", action="store_true", help="launch the step eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--scaled-only", action="store_true", help="only time draft/accept on the bandwidth-sized batches (a short run to profile those kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     args.steps = max(args.steps, 1)
@@ -818,6 +819,11 @@ def main():
     dev = torch.device("cuda", local_rank)
     pk = peaks()
 
+    if args.scaled_only:
+        head = Head(torch, ngs, c, dev, pk, time_table=False)
+        print(json.dumps({"scaled_streams": scaled_streams(head.ctx, torch, dev, c, pk), "workload_head": workload_string(c)}))
+        head.ctx.close()
+        return 0
     names = [args.workload] + ([] if args.no_per_config else [n for n in ("C2", "C3", "C4", "C5") if n != args.workload and args.workload != "C1"])
     heads, per_config, head_rec, head_x = {}, {}, None, None
     for name in names:
