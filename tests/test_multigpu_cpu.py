@@ -144,3 +144,18 @@ def test_two_gloo_ranks_stitch_their_table_slices_into_the_whole_table():
     # single process: the slice is the table
     one = multigpu.all_gather_rows(torch.from_numpy(whole), 37, 0, 1)
     assert one.numpy().tolist() == whole.tolist()
+
+
+def test_bench_refuses_to_run_fewer_ranks_than_asked():
+    """`bench.py --gpus N` without a launcher starts N ranks itself - and fails loudly when the machine does not
+    show N GPUs (here: none), instead of quietly running one rank."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "1"], capture_output=True, text=True,
+                       env=env, timeout=300)
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 2:
+        return                                             # a machine with two GPUs would simply run it
+    assert r.returncode != 0
+    assert "refusing to run fewer ranks than asked" in (r.stderr + r.stdout)
