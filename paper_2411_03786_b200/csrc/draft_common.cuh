@@ -60,11 +60,19 @@ __device__ __forceinline__ int cont_tok(const int32_t* __restrict__ h, int Lw, i
     if (Lw != 0 && i >= Lw) i = p + t % (Lw - p);
     return h[i];
 }
+// The same with the variant fixed at compile time: the grouping of matches is bound by instructions, and the
+// plain rule should not carry the other one's tests (they cost the batch kernels a third of their time).
+template <bool PT>
+__device__ __forceinline__ int cont_tok_t(const int32_t* __restrict__ h, int Lw, int p, int t) {
+    if constexpr (PT) return cont_tok(h, Lw, p, t);
+    else return h[p + t];
+}
 
 // Group the match whose continuation starts at p (query index qi) in an open-addressing table:
 // rep[slot] = (qi << 28 | start of the group's first-seen continuation), cnt, last; a collision is
 // resolved by comparing the actual tokens, so grouping is exact.  n_groups / overflow are the table's
 // counters; once overflow is set the pass is void and nothing more is inserted.
+template <bool PT = false>
 __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int p, int qi, int key_len, uint32_t hsh,
                                              int slots, int max_groups, int* rep, int* cnt, int* last,
                                              int* grp_slot, int* n_groups, int* overflow, int Lw = 0) {
@@ -92,7 +100,7 @@ __device__ __forceinline__ void insert_match(const int32_t* __restrict__ h, int 
             const int rp = cur & 0x0FFFFFFF;
             bool same = true;
             for (int t = 0; t < key_len; ++t)
-                if (cont_tok(h, Lw, rp, t) != cont_tok(h, Lw, p, t)) {
+                if (cont_tok_t<PT>(h, Lw, rp, t) != cont_tok_t<PT>(h, Lw, p, t)) {
                     same = false;
                     break;
                 }
@@ -160,14 +168,14 @@ __device__ __forceinline__ void model_chain(const DraftParams& P, int x, int lan
 // needs overlap.  No barrier inside: the caller synchronises before (table cleared) and after.
 // Returns how many vectors of the history the calling warp had gone past when it stopped (all of them unless
 // the table overflowed): the caller sizes the next round of passes from it.
-template <int U = 4>  // 128-bit loads a thread keeps in flight
+template <int U = 4, bool PT = false>  // U: 128-bit loads a thread keeps in flight; PT: SPEC_FLAG_PARTIAL_TAIL (the caller passes what P.flags says)
 __device__ __forceinline__ int scan_pass(const DraftParams& P, const int32_t* __restrict__ h, int L, int R, int r,
                                           int t0, int t1, int t2, int t3, const DraftTable& T, int* wq, int tid, int nthr) {
     const int w = P.w, lane = tid & 31;
     const int n_scan = L - w;  // token index x = p - 1 runs over [0, n_scan)
     const int key_len = (P.flags & SPEC_FLAG_KEY_NEXT_TOKEN) ? 1 : w;
     const bool need2 = P.q_min >= 2;  // every query has at least two tokens: test the second one in registers
-    const bool partial = (P.flags & SPEC_FLAG_PARTIAL_TAIL) != 0;  // occurrences with fewer than w following tokens count too
+    constexpr bool partial = PT;  // occurrences with fewer than w following tokens count too
     const int Lw = partial ? L : 0;
     const int4* h4 = reinterpret_cast<const int4*>(h);
     const int n_vec = (max(n_scan, 0) + 3) >> 2;
@@ -196,13 +204,13 @@ __device__ __forceinline__ int scan_pass(const DraftParams& P, const int32_t* __
         }
         const int p = x + 1;
         uint32_t hc = 0x9E3779B9u;  // one multiply-add per token, mixed once per query length below
-        for (int t = 0; t < key_len; ++t) hc = hc * 0x85EBCA6Bu + (uint32_t)cont_tok(h, Lw, p, t);
+        for (int t = 0; t < key_len; ++t) hc = hc * 0x85EBCA6Bu + (uint32_t)cont_tok_t<PT>(h, Lw, p, t);
         for (int qi = 0; qi < P.n_q; ++qi) {
             const int q = P.qs[qi];
             if (m < q || (!partial && L < q + w)) continue;
             const uint32_t hq = fmix32(hc + (uint32_t)qi * 0x632BE5ABu);
             if (R > 1 && (int)(fmix32(hq ^ 0xA511E9B3u) % (uint32_t)R) != r) continue;
-            insert_match(h, p, qi, key_len, hq, P.slots, P.max_groups, T.rep, T.cnt, T.last, T.grp_slot, T.n_groups, T.overflow, Lw);
+            insert_match<PT>(h, p, qi, key_len, hq, P.slots, P.max_groups, T.rep, T.cnt, T.last, T.grp_slot, T.n_groups, T.overflow, Lw);
         }
     };
     int qn = 0;  // queued matches (the same in every lane)

@@ -81,6 +81,7 @@ __device__ __forceinline__ void named_arrive(int id, int count) {
     asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
+template <bool PT>  // PT: SPEC_FLAG_PARTIAL_TAIL
 __global__ void __launch_bounds__(STREAM_THREADS, 1) draft_stream_kernel(const DraftParams P, const StreamLayout Y, unsigned int* work) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     StreamMisc* sm = reinterpret_cast<StreamMisc*>(smem_raw + Y.misc);
@@ -111,7 +112,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) draft_stream_kernel(const D
             named_arrive(BAR_FEMPTY + k, FETCH_COUNT);
             k ^= 1;
             const int32_t* __restrict__ h = P.hist + (size_t)s * P.cap;
-            const bool partial = (P.flags & SPEC_FLAG_PARTIAL_TAIL) != 0;
+            constexpr bool partial = PT;
             bool any_q = false;
             for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + (partial ? 1 : P.w));
             const bool scan = any_q && (L - P.w >= 1 || (partial && L >= 2));
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) draft_stream_kernel(const D
                         sm->desc[buf].flags = (r == 0 ? PASS_FIRST : 0) | ((r == R - 1 || gave_up) ? PASS_LAST : 0) | (gave_up ? PASS_GAVE_UP : 0);
                     }
                     int reached = 0;
-                    if (scan && !gave_up) reached = scan_pass<STREAM_LOADS>(P, h, L, R, r, t0, t1, t2, t3, T, wq, tid, SWT);
+                    if (scan && !gave_up) reached = scan_pass<STREAM_LOADS, PT>(P, h, L, R, r, t0, t1, t2, t3, T, wq, tid, SWT);
                     if (tid == 0) sm->reached = reached;
                     named_sync(BAR_SCAN, SWT);  // every scanner's matches are in the table
                     overflowed = *((volatile int*)T.overflow) != 0;
@@ -281,18 +282,20 @@ int launch_draft_stream(spec_ctx* ctx, DraftParams& P, cudaStream_t st) {
     Y.misc = off;
     off += round_up16((int)sizeof(StreamMisc));
     Y.bytes = off;  // at most about 190 KB (largest draft shape)
+    const int pt = (P.flags & SPEC_FLAG_PARTIAL_TAIL) ? 1 : 0;
+    void (*kern)(const DraftParams, const StreamLayout, unsigned int*) = pt ? draft_stream_kernel<true> : draft_stream_kernel<false>;
     {
-        static bool attr_set[64] = {};
+        static bool attr_set[64][2] = {};
         std::lock_guard<std::mutex> lock(host_mutex());
-        if (!attr_set[ctx->device & 63]) {
-            int rc = check_cuda(ctx, cudaFuncSetAttribute(draft_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024),
+        if (!attr_set[ctx->device & 63][pt]) {
+            int rc = check_cuda(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024),
                                 "draft (long histories): cudaFuncSetAttribute");
             if (rc) return rc;
-            attr_set[ctx->device & 63] = true;
+            attr_set[ctx->device & 63][pt] = true;
         }
     }
     const int grid = P.S < ctx->num_sms ? P.S : ctx->num_sms;
-    cudaError_t e = launch_pdl(draft_stream_kernel, dim3((unsigned)grid), dim3(STREAM_THREADS), (size_t)Y.bytes, st, P, Y, ctx->d_draft_work);
+    cudaError_t e = launch_pdl(kern, dim3((unsigned)grid), dim3(STREAM_THREADS), (size_t)Y.bytes, st, P, Y, ctx->d_draft_work);
     ctx->launches += 1;
     return check_cuda(ctx, e, "draft_context_ngrams (long histories) launch");
 }

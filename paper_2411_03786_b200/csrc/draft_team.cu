@@ -62,7 +62,7 @@ struct TeamMisc {
     unsigned long long tau[kMaxNQ];
 };
 
-template <int T>
+template <int T, bool PT>  // T warps per team; PT: SPEC_FLAG_PARTIAL_TAIL
 __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(const DraftParams P, const TeamLayout Y, unsigned int* work) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr int TT = T * 32;  // threads of a team
@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(cons
         // ---- context N-grams
         const int n_scan = L - P.w;
         const int t0 = sm->tq[0], t1 = sm->tq[1], t2 = sm->tq[2], t3 = sm->tq[3];
-        const bool partial = (P.flags & SPEC_FLAG_PARTIAL_TAIL) != 0;
+        constexpr bool partial = PT;
         bool any_q = false;
         for (int qi = 0; qi < P.n_q; ++qi) any_q = any_q || (L >= P.qs[qi] + (partial ? 1 : P.w));
         int R = 1;
@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(cons
                     sm->overflow = 0;
                 }
                 team_sync();
-                const int reached = scan_pass(P, h, L, R, r, t0, t1, t2, t3, tab, wq, tid, TT);
+                const int reached = scan_pass<4, PT>(P, h, L, R, r, t0, t1, t2, t3, tab, wq, tid, TT);
                 if (tid == 0) sm->reached = reached;
                 team_sync();  // the team's matches are in the table
                 if (*((volatile int*)&sm->overflow)) {
@@ -270,12 +270,16 @@ int launch_draft_team(spec_ctx* ctx, DraftParams& P, cudaStream_t st) {
     }
     if (Y.teams < 1) return kDraftNoFit;
     const size_t smem = (size_t)Y.teams * Y.bytes;
-    void (*kern)(const DraftParams, const TeamLayout, unsigned int*) =
-        T == 1 ? draft_team_kernel<1> : T == 2 ? draft_team_kernel<2> : T == 4 ? draft_team_kernel<4> : T == 8 ? draft_team_kernel<8>
-                                                                                                            : draft_team_kernel<16>;
+    using Kern = void (*)(const DraftParams, const TeamLayout, unsigned int*);
+    static const Kern kerns[2][5] = {
+        {draft_team_kernel<1, false>, draft_team_kernel<2, false>, draft_team_kernel<4, false>, draft_team_kernel<8, false>, draft_team_kernel<16, false>},
+        {draft_team_kernel<1, true>, draft_team_kernel<2, true>, draft_team_kernel<4, true>, draft_team_kernel<8, true>, draft_team_kernel<16, true>}};
+    const int pt = (P.flags & SPEC_FLAG_PARTIAL_TAIL) ? 1 : 0;
+    const int ti0 = T == 1 ? 0 : T == 2 ? 1 : T == 4 ? 2 : T == 8 ? 3 : 4;
+    const Kern kern = kerns[pt][ti0];
     {
-        static bool attr_set[64][5] = {};
-        const int ti = T == 1 ? 0 : T == 2 ? 1 : T == 4 ? 2 : T == 8 ? 3 : 4;
+        static bool attr_set[64][10] = {};
+        const int ti = pt * 5 + ti0;
         std::lock_guard<std::mutex> lock(host_mutex());
         if (!attr_set[ctx->device & 63][ti]) {
             int rc = check_cuda(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TEAM_SMEM_BUDGET),
