@@ -217,7 +217,7 @@ def scaled_streams(ctx, torch, dev, c, pk):
         ms = timed(lambda: ctx.draft_context_ngrams(hist, lens, qs, topk, B, w, out=bufs), reps)
         by = 4.0 * S * L + 4.0 * S * B * (w + 2) + 8.0 * S
         ix_ms = None
-        if L >= 131072 and not tag:   # the same batch drafted from the incremental context index (built once, outside the timing)
+        if not tag:   # the same batch drafted from the incremental context index (built once, outside the timing)
             index = ctx.context_index_build(hist, lens, qs, w)
             ix_ms = timed(lambda: ctx.draft_context_ngrams_indexed(index, hist, lens, qs, topk, B, w, out=bufs), reps)
             del index
