@@ -26,7 +26,7 @@ struct DraftParams {
     int32_t* counts;
     int* status;
     int slots;       // hash table size (power of two)
-    int max_groups;  // slots / 2
+    int max_groups;  // groups one pass may open: half to three quarters of the slots
     int stage_hist;  // latency kernel: 1 = copy the history into shared memory first (single CTA, short history)
     int hist_off;    // where that copy lives, in ints from the start of the hash table
 };

@@ -204,21 +204,28 @@ static int round_up16(int x) { return (x + 15) & ~15; }
 
 int launch_draft_team(spec_ctx* ctx, DraftParams& P, cudaStream_t st) {
     const int sms = ctx->num_sms;
-    // Table: twice as many slots as groups are expected.  A query of one token matches up to a tenth of the
-    // positions on natural token statistics, longer queries around one in a hundred.  (A table that
-    // overflows costs whole rescans - measured on 4096 x 2048 tokens with a one-token query: 128 us with 512
-    // slots, 80 us with 1024 - so the estimate errs on the large side.)
-    const int expect = P.q_min >= 2 || P.n_q == 0 ? P.cap / 72 : P.cap / 4;
+    // Table: filled to at most three quarters (groups are found by linear probing from a mixed hash).  A query
+    // of one token matches up to a tenth of the positions on natural token statistics and most of those
+    // matches differ in their continuation (cap / 8 groups at the most on Zipf 1.1 over 32000 tokens), longer
+    // queries around one in a hundred.  A table that overflows costs whole rescans, a larger table costs
+    // sequences in flight (it is most of a team's shared memory): 4096 x 2048 tokens with a one-token query
+    // take 128 us with 256 groups, 80 us with 512 groups in 1024 slots and less again with 384 groups in 512.
+    const int expect = P.q_min >= 2 || P.n_q == 0 ? P.cap / 72 : P.cap / 6;
     int slots = 256;
-    while (slots < expect && slots < 2048) slots <<= 1;
+    while (slots / 4 * 3 < expect && slots < 2048) slots <<= 1;
     P.slots = slots;
-    P.max_groups = slots / 2;
+    P.max_groups = slots / 4 * 3;
     P.stage_hist = 1;
     P.hist_off = 0;
     // warps per team: enough teams per SM (of its 32 warps) to hold the batch's share of sequences
     const int per_sm = (P.S + sms - 1) / sms;
     int T = 16;
     while (T > 1 && 32 / T < per_sm) T >>= 1;
+    // ... but at least a warp per 512 tokens of history (measured: 1024 tokens run best with two warps, 2048 with
+    // four; a scan spread thinner leaves the sequence's serial phases to too few threads)
+    int t_len = 1;
+    while (t_len < 16 && t_len * 2 * 512 <= P.cap) t_len <<= 1;
+    if (T < t_len) T = t_len;
 #ifdef NGRAM_SPEC_TUNING
     if (const char* ov = getenv("NGRAM_SPEC_TEAM")) {  // tuning builds only: warps per team
         const int t = atoi(ov);
@@ -228,7 +235,7 @@ int launch_draft_team(spec_ctx* ctx, DraftParams& P, cudaStream_t st) {
         const int t = atoi(ov);
         if (t >= 64 && t <= 4096 && (t & (t - 1)) == 0) {
             P.slots = t;
-            P.max_groups = t / 2;
+            P.max_groups = t / 4 * 3;
         }
     }
 #endif
