@@ -66,8 +66,10 @@ template <int T, bool PT>  // T warps per team; PT: SPEC_FLAG_PARTIAL_TAIL
 __global__ void __launch_bounds__(TEAM_MAX_WARPS * 32, 2) draft_team_kernel(const DraftParams P, const TeamLayout Y, unsigned int* work) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr int TT = T * 32;  // threads of a team
-    const int team = (int)threadIdx.x / TT, tid = (int)threadIdx.x % TT;
-    const int lane = tid & 31, warp = tid >> 5;
+    // A team's warps are Y.teams apart: with four or eight teams per CTA they all sit on the same scheduler of
+    // the SM and, running the same phase of the same sequence, share the instruction lines it has fetched.
+    const int team = ((int)threadIdx.x >> 5) % Y.teams, warp = ((int)threadIdx.x >> 5) / Y.teams;
+    const int lane = (int)threadIdx.x & 31, tid = warp * 32 + lane;
     unsigned char* base = smem_raw + (size_t)team * Y.bytes;
     TeamMisc* sm = reinterpret_cast<TeamMisc*>(base + Y.misc);
     DraftTable tab;
