@@ -15,9 +15,10 @@
 // therefore owns one row of A and walks its columns in ascending vocabulary order, which makes
 // "lowest token id wins ties" a matter of using a strict comparison.
 //
-// Work is cut into units (m_tile, vocabulary chunk).  CTA b of the grid = group x slots works on
-// m-tile b % group of each m-group and on chunks b / group, + slots, ...: CTAs of one slot walk
-// the same chunks of W together, so W comes from HBM once per m-group.  Inside a unit the CTA
+// Work is cut into units (m_tile, vocabulary chunk), numbered so that consecutive units are the m-tiles
+// of one m-group on the same chunk, and dealt out round-robin over the CTAs: the CTAs at work at any
+// moment walk the same few chunks of W together, so W comes from HBM once per m-group, and every SM
+// has work until the last round.  Inside a unit the CTA
 // sweeps the chunk in tiles of up to 256 columns and keeps the running
 // reduction in registers, then flushes once: a 64-bit atomicMax of (value, ~index) for the arg
 // max, a partial list for the top-k.  Small M (memory-bound: every SM streams its own slice of
@@ -64,7 +65,7 @@ struct GemmParams {
     int n_chunks;  // vocabulary chunks per m-tile
     int group;     // m-tiles that run side by side on the same W chunk (L2 reuse)
     int n_groups;  // ceil(n_mtiles / group)
-    int n_slots;   // grid = group * n_slots
+    int n_slots;   // slot order: grid = group * n_slots; 0 = round-robin order (see UnitIter)
     int a_box_rows;   // rows of A per TMA box (128, or fewer when A has fewer rows)
     int a2_rows;      // dual: rows of the second m-tile's TMA box (its own tensor map)
     int a_bytes;      // shared-memory bytes reserved for the A tile of a stage (multiple of 1024)
@@ -255,19 +256,43 @@ __device__ __forceinline__ void chunk_argmax(const float (&v)[32], float& best, 
 struct Unit {
     int m_tile, chunk, box_begin, box_end;
 };
-// Units of this CTA in execution order.
+// Units of this CTA in execution order.  Two orders:
+//  - slots (chunks that cost a partial result per row and are therefore few and long - top-k lists, sums of
+//    squares): the grid is group x n_slots CTAs, CTA b works on m-tile b % group of each m-group and on chunks
+//    b / group, + n_slots, ...; the CTAs of one slot start a chunk together and walk its tiles in step, so W
+//    comes from HBM once per m-group;
+//  - round-robin (n_slots = 0; the arg max, whose chunks are single tiles): the launch's units are numbered
+//    m-group by m-group, inside a group chunk by chunk, inside a chunk m-tile by m-tile, and CTA b takes units
+//    b, b + grid, b + 2 grid, ...  Units cost the same, so every SM is busy until the last round whatever
+//    the numbers of m-tiles and chunks, and the CTAs at work at any moment hold consecutive units - the
+//    m-tiles of a group on the same few tiles of W.
 struct UnitIter {
-    int mg, c, mi, slot;
+    long long u;          // round-robin: the next unit
+    int mg, c, mi, slot;  // slots: m-group, chunk, m-tile in the group, slot
     __device__ __forceinline__ explicit UnitIter(const GemmParams& p)
-        : mg(0), c((int)blockIdx.x / p.group), mi((int)blockIdx.x % p.group), slot((int)blockIdx.x / p.group) {}
-    __device__ __forceinline__ bool next(const GemmParams& p, Unit& u) {
+        : u((long long)blockIdx.x), mg(0), c((int)blockIdx.x / p.group), mi((int)blockIdx.x % p.group), slot((int)blockIdx.x / p.group) {}
+    __device__ __forceinline__ bool next(const GemmParams& p, Unit& un) {
+        if (p.n_slots == 0) {
+            if (u >= (long long)p.n_chunks * p.n_mtiles) return false;
+            const long long per_group = (long long)p.n_chunks * p.group;  // units of a full m-group (only the last can be ragged)
+            const int g = (int)(u / per_group);
+            const int r = (int)(u - (long long)g * per_group);
+            const int gm = min(p.group, p.n_mtiles - g * p.group);  // m-tiles of this group
+            const int cc = r / gm;
+            un.m_tile = g * p.group + (r - cc * gm);
+            un.chunk = cc;
+            un.box_begin = (int)((long long)cc * p.n_boxes / p.n_chunks);
+            un.box_end = (int)((long long)(cc + 1) * p.n_boxes / p.n_chunks);
+            u += (long long)gridDim.x;
+            return true;
+        }
         while (mg < p.n_groups) {
             const int m_tile = mg * p.group + mi;
             if (m_tile < p.n_mtiles && c < p.n_chunks) {
-                u.m_tile = m_tile;
-                u.chunk = c;
-                u.box_begin = (int)((long long)c * p.n_boxes / p.n_chunks);
-                u.box_end = (int)((long long)(c + 1) * p.n_boxes / p.n_chunks);
+                un.m_tile = m_tile;
+                un.chunk = c;
+                un.box_begin = (int)((long long)c * p.n_boxes / p.n_chunks);
+                un.box_end = (int)((long long)(c + 1) * p.n_boxes / p.n_chunks);
                 c += p.n_slots;
                 return true;
             }
@@ -795,7 +820,6 @@ static void finish_shape(Shape& sh, int a_rows, int V) {
     const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
     sh.box_idx = sh.box_n == 16 ? 0 : sh.box_n == 32 ? 1 : sh.box_n == 64 ? 2 : sh.box_n == 128 ? 3 : 4;
     sh.n_groups = sh.dual ? 1 : (n_mtiles + sh.group - 1) / sh.group;
-    sh.n_slots = sh.grid / sh.group;
     const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
     const int chunk_max = (n_boxes + sh.n_chunks - 1) / sh.n_chunks;
     const int nb_max = std::min(TILE_N / sh.box_n, chunk_max);
@@ -814,11 +838,13 @@ static void finish_shape(Shape& sh, int a_rows, int V) {
 // Unit shapes.  `box_n` is the granularity in which the vocabulary is cut into chunks and tiles (a
 // tile is then copied in power-of-two pieces, see the producer).  One m-tile (memory-bound): every
 // SM streams its own slice of W once, cut to 32 rows so slices balance to within 32 rows.  Several
-// m-tiles (tensor-bound): `group` m-tiles share each W chunk, tiles are whole 256-row blocks (one
-// copy per k-block) and every slot sweeps one chunk per m-group.  (Measured on B200, V=32000,
-// d=4096, when a tile was still copied box by box: 32-row boxes 0.9, 64-row 1.1, 256-row
-// 1.2 PFLOP/s; groups of 8..16 beat groups of 2..4 by 10-20%.)
-static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks, bool allow_dual) {
+// m-tiles (tensor-bound): `group` m-tiles share each W chunk and tiles are whole 256-row blocks (one
+// copy per k-block).  (Measured on B200, V=32000, d=4096, when a tile was still copied box by box:
+// 32-row boxes 0.9, 64-row 1.1, 256-row 1.2 PFLOP/s; groups of 8..16 beat groups of 2..4 by 10-20%.)
+// `tile_chunks`: a chunk is a single tile (the arg max is merged per row with one atomic per unit, so
+// units may be as small as a tile and the round-robin then balances to within one tile); otherwise a chunk
+// costs a partial result per row (top-k lists, sums of squares) and there are about #SMs / group of them.
+static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks, bool allow_dual, bool tile_chunks) {
     const int n_mtiles = (a_rows + BLOCK_M - 1) / BLOCK_M;
     Shape sh{};
     if (n_mtiles == 1 || (n_mtiles == 2 && allow_dual)) {
@@ -829,32 +855,50 @@ static Shape choose_shape(int a_rows, int V, int sms, size_t max_chunks, bool al
         sh.n_chunks = (int)std::min<size_t>((size_t)std::min(sms, (V + 31) / 32), max_chunks);
         sh.grid = sh.n_chunks;
     } else {
-        // the group (up to 16 m-tiles) that keeps most SMs busy, counting a ragged last m-group;
-        // larger groups re-stream W less often
-        double best = -1.0;
-        for (int g = std::min(16, n_mtiles); g >= 1; --g) {
-            const int slots = sms / g, groups = (n_mtiles + g - 1) / g;
-            const double busy = (double)n_mtiles / (groups * g) * (double)(slots * g) / sms * (1.0 - 0.02 * (16 - g));
-            if (busy > best + 1e-9) {
-                best = busy;
-                sh.group = g;
+        if (tile_chunks) {
+            // round-robin order: neither the group nor the number of chunks has to divide the number of SMs;
+            // larger groups re-stream W less often
+            // (measured, V = 128256, 22 m-tiles: groups of 8 / 11 / 16 / 22 run at 1249 / 1268 / 1286 / 1290 TFLOP/s;
+            // V = 32000, 72 m-tiles: groups of 16 / 24 / 36 / 72 at 1267 / 1310 / 1326 / 1206 - beyond some thirty
+            // m-tiles the hidden states of a group and the tiles of W in flight no longer share the L2)
+            const int n_groups = (n_mtiles + 31) / 32;
+            sh.group = (n_mtiles + n_groups - 1) / n_groups;
+            sh.box_n = 256;
+            while (sh.box_n > 32 && (long long)((V + sh.box_n - 1) / sh.box_n) * n_mtiles < sms) sh.box_n >>= 1;
+            const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
+            const int tiles = (int)(((long long)n_boxes * sh.box_n + TILE_N - 1) / TILE_N);  // one tile per chunk
+            sh.n_chunks = (int)std::min<size_t>((size_t)std::min(tiles, n_boxes), max_chunks);
+            sh.grid = (int)std::min<long long>((long long)sms, (long long)sh.n_chunks * n_mtiles);
+            sh.n_slots = 0;
+        } else {
+            // slot order: the group (up to 16 m-tiles) that keeps most SMs busy, counting a ragged last m-group;
+            // larger groups re-stream W less often
+            double best = -1.0;
+            for (int g = std::min(16, n_mtiles); g >= 1; --g) {
+                const int slots = sms / g, groups = (n_mtiles + g - 1) / g;
+                const double busy = (double)n_mtiles / (groups * g) * (double)(slots * g) / sms * (1.0 - 0.02 * (16 - g));
+                if (busy > best + 1e-9) {
+                    best = busy;
+                    sh.group = g;
+                }
             }
+            const int slots = sms / sh.group;
+            // 256-row boxes need one TMA issue per k-block and measured faster than better balanced chunks
+            // of smaller boxes; fall back to smaller boxes only when the vocabulary is too small to give
+            // every slot a chunk
+            sh.box_n = 256;
+            while (sh.box_n > 32 && (V + sh.box_n - 1) / sh.box_n < slots) sh.box_n >>= 1;
+            const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
+            sh.n_chunks = (int)std::min<size_t>((size_t)std::min(slots, n_boxes), max_chunks);
+            sh.n_slots = std::min(slots, sh.n_chunks);
+            sh.grid = sh.group * sh.n_slots;
         }
-        const int slots = sms / sh.group;
-        // 256-row boxes need one TMA issue per k-block and measured faster than better balanced chunks
-        // of smaller boxes; fall back to smaller boxes only when the vocabulary is too small to give
-        // every slot a chunk
-        sh.box_n = 256;
-        while (sh.box_n > 32 && (V + sh.box_n - 1) / sh.box_n < slots) sh.box_n >>= 1;
-        const int n_boxes = (V + sh.box_n - 1) / sh.box_n;
-        sh.n_chunks = (int)std::min<size_t>((size_t)std::min(slots, n_boxes), max_chunks);
-        sh.grid = sh.group * std::min(slots, sh.n_chunks);
     }
     finish_shape(sh, a_rows, V);
     return sh;
 }
 
-static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks, bool allow_dual = false) {
+static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks, bool allow_dual = false, bool tile_chunks = false) {
 #ifdef NGRAM_SPEC_TUNING
     // Tuning builds only: NGRAM_SPEC_SHAPE="box,group,chunks" overrides the choice (values are clamped).
     if (const char* ov = getenv("NGRAM_SPEC_SHAPE")) {
@@ -866,24 +910,24 @@ static Shape cached_shape(spec_ctx* ctx, int a_rows, size_t max_chunks, bool all
             s.group = std::max(1, std::min(std::min(g, n_mtiles), ctx->num_sms));
             const int n_boxes = (ctx->V + box - 1) / box;
             s.n_chunks = (int)std::max<size_t>(1, std::min<size_t>(std::min<size_t>((size_t)std::max(c, 1), (size_t)n_boxes), max_chunks));
-            s.grid = s.group * std::min(ctx->num_sms / s.group, s.n_chunks);
+            s.grid = (int)std::min<long long>((long long)ctx->num_sms, (long long)s.n_chunks * (s.dual ? 1 : n_mtiles));
             finish_shape(s, a_rows, ctx->V);
             return s;
         }
     }
 #endif
     // Process-wide table of the shapes chosen so far.
-    const auto key = std::make_tuple(a_rows, ctx->V, ctx->d, ctx->num_sms, max_chunks, allow_dual);
+    const auto key = std::make_tuple(a_rows, ctx->V, ctx->d, ctx->num_sms, max_chunks, allow_dual, tile_chunks);
     std::lock_guard<std::mutex> lock(host_mutex());
-    static std::map<std::tuple<int, int, int, int, size_t, bool>, Shape> cache;
+    static std::map<std::tuple<int, int, int, int, size_t, bool, bool>, Shape> cache;
     auto it = cache.find(key);
     if (it != cache.end()) return it->second;
-    Shape s = choose_shape(a_rows, ctx->V, ctx->num_sms, max_chunks, allow_dual);
+    Shape s = choose_shape(a_rows, ctx->V, ctx->num_sms, max_chunks, allow_dual, tile_chunks);
     cache[key] = s;
 #ifdef NGRAM_SPEC_TUNING
     if (getenv("NGRAM_SPEC_TRACE"))
-        fprintf(stderr, "[ngram_spec] rows=%d V=%d d=%d: dual=%d box=%d group=%d slots=%d chunks=%d grid=%d a_box=%d stages=%d stage=%dB smem=%dB\n",
-                a_rows, ctx->V, ctx->d, s.dual, s.box_n, s.group, s.n_slots, s.n_chunks, s.grid, s.a_box_rows, s.stages, s.stage_bytes, s.smem);
+        fprintf(stderr, "[ngram_spec] rows=%d V=%d d=%d: dual=%d box=%d group=%d groups=%d chunks=%d grid=%d a_box=%d stages=%d stage=%dB smem=%dB\n",
+                a_rows, ctx->V, ctx->d, s.dual, s.box_n, s.group, s.n_groups, s.n_chunks, s.grid, s.a_box_rows, s.stages, s.stage_bytes, s.smem);
 #endif
     return s;
 }
@@ -955,7 +999,7 @@ int launch_verify(spec_ctx* ctx, const void* d_hidden, int M, int32_t* d_argmax,
                   const AcceptArgs* fuse, long long* d_keys_out, int idx_offset) {
     int rc = set_smem_attr<MODE_ARGMAX, 1>(ctx);
     if (rc) return rc;
-    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
+    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true, true);
     const WMaps* tmW;
     if ((rc = w_map(ctx, &tmW))) return rc;
     const CUtensorMap* tmA;
@@ -1041,7 +1085,7 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
                       cudaStream_t st) {
     int rc = set_smem_attr<MODE_ARGMAX_Q8, 1>(ctx);
     if (rc) return rc;
-    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true);
+    const Shape sh = cached_shape(ctx, M, (size_t)1 << 20, true, true);
     if (!ctx->tm_q_ready) {
         if ((rc = make_w_maps(ctx, &ctx->tm_q, ctx->wq, 1))) return rc;
         ctx->tm_q_ready = true;
@@ -1070,7 +1114,7 @@ int launch_verify_fp8(spec_ctx* ctx, const uint8_t* d_hq, const float* d_hscale,
 int launch_logits(spec_ctx* ctx, const void* d_rows, int m, float* d_logits, cudaStream_t st) {
     int rc = set_smem_attr<MODE_STORE, 1>(ctx);
     if (rc) return rc;
-    const Shape sh = cached_shape(ctx, m, (size_t)1 << 20);
+    const Shape sh = cached_shape(ctx, m, (size_t)1 << 20, false, true);
     const WMaps* tmW;
     if ((rc = w_map(ctx, &tmW))) return rc;
     CUtensorMap tmA;
